@@ -1,0 +1,203 @@
+"""fp64 CPU oracle of the BASP attention layer -- TEST INFRASTRUCTURE ONLY.
+
+Thin numpy/ctypes front end of ``basp_oracle.c`` (plain C, fp64, literal loops of the
+paper's definitions: Algorithm 1, Algorithm 2, the two group-local all-to-alls of
+Section IV-C and the attention equation of Section II-A with a causal mask).
+
+Nothing here is imported by the CUDA package; only the tests, the smoke check and the
+benchmark's CPU-baseline leg may use it.  It shares no code with the CUDA path.
+
+Conventions
+-----------
+* bf16 tensors are numpy ``uint16`` arrays holding the bit patterns.
+* ``seq`` arenas are ``[N, Bl, T, H, D]``, ``head`` arenas ``[N, Bl, S, H/K, D]``.
+* ``G = 0`` (or ``G = B``) is BASP, ``G = 1`` is standard Ulysses.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "basp_oracle.c")
+_LIB = os.path.join(_HERE, "libbasp_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP, strict IEEE: no -ffast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-march=native", "-fopenmp", "-fno-fast-math", "-shared", "-fPIC",
+               "-o", _LIB, _SRC, "-lm"]
+        try:
+            subprocess.check_call(cmd)
+        except subprocess.CalledProcessError:
+            cmd.remove("-march=native")
+            subprocess.check_call(cmd)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB)
+        _lib.oracle_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+# ----------------------------------------------------------------------------- plan
+@dataclass(frozen=True)
+class Plan:
+    N: int      # ranks
+    B: int      # micro-batch (sequences)
+    G: int      # groups
+    K: int      # ranks per group
+    Bl: int     # sequences per group
+    S: int      # tokens per sequence
+    T: int      # tokens per rank and sequence
+
+    def group_ranks(self, g: int) -> list[int]:
+        out = (ctypes.c_int * self.K)()
+        _load().oracle_group_ranks(self.K, g, out)
+        return list(out)
+
+    def rank_info(self, r: int, Hq: int, Hkv: int) -> dict:
+        out = (ctypes.c_int * 10)()
+        _load().oracle_rank_info(self.K, self.Bl, self.T, Hq, Hkv, r, out)
+        keys = ("group", "local_rank", "seq_begin", "seq_end", "token_begin", "token_end",
+                "q_head_begin", "q_head_end", "kv_head_begin", "kv_head_end")
+        return dict(zip(keys, list(out)))
+
+
+def plan(N: int, B: int, S: int, G: int = 0) -> Plan:
+    """Algorithm 1 (+ the explicit group count of Section IV-C).  Raises ValueError
+    where the paper asserts or declares the case unsupported."""
+    out = (ctypes.c_int * 4)()
+    rc = _load().oracle_plan(int(N), int(B), int(G), int(S), out)
+    if rc != 0:
+        raise ValueError(f"invalid BASP plan N={N} B={B} G={G} S={S}")
+    K, G_, Bl, T = list(out)
+    return Plan(N=N, B=B, G=G_, K=K, Bl=Bl, S=S, T=T)
+
+
+# ------------------------------------------------------------------ permutations
+def _esize(a: np.ndarray) -> int:
+    return int(a.dtype.itemsize)
+
+
+def partition(X: np.ndarray, pl: Plan) -> np.ndarray:
+    """Algorithm 2 for every rank: X[B,S,H,D] -> [N,Bl,T,H,D]."""
+    X = np.ascontiguousarray(X)
+    B, S, H, D = X.shape
+    assert B == pl.B and S == pl.S
+    out = np.empty((pl.N, pl.Bl, pl.T, H, D), dtype=X.dtype)
+    _load().oracle_partition(_p(X), _p(out), pl.N, pl.K, pl.Bl, S, H, D, _esize(X))
+    return out
+
+
+def gather(shards: np.ndarray, pl: Plan) -> np.ndarray:
+    """Inverse of :func:`partition`: [N,Bl,T,H,D] -> X[B,S,H,D]."""
+    shards = np.ascontiguousarray(shards)
+    N, Bl, T, H, D = shards.shape
+    out = np.empty((pl.B, pl.S, H, D), dtype=shards.dtype)
+    _load().oracle_gather(_p(shards), _p(out), pl.N, pl.K, pl.Bl, pl.S, H, D, _esize(shards))
+    return out
+
+
+def s2h(seq: np.ndarray, pl: Plan) -> np.ndarray:
+    """Group-local all-to-all, sequence-sharded -> head-sharded (Section IV-C)."""
+    seq = np.ascontiguousarray(seq)
+    N, Bl, T, H, D = seq.shape
+    assert (N, Bl, T) == (pl.N, pl.Bl, pl.T) and H % pl.K == 0
+    out = np.empty((N, Bl, pl.S, H // pl.K, D), dtype=seq.dtype)
+    _load().oracle_s2h(_p(seq), _p(out), N, pl.K, Bl, pl.S, H, D, _esize(seq))
+    return out
+
+
+def h2s(head: np.ndarray, pl: Plan) -> np.ndarray:
+    """Group-local all-to-all, head-sharded -> sequence-sharded (the reverse one)."""
+    head = np.ascontiguousarray(head)
+    N, Bl, S, Hl, D = head.shape
+    assert (N, Bl, S) == (pl.N, pl.Bl, pl.S)
+    out = np.empty((N, Bl, pl.T, Hl * pl.K, D), dtype=head.dtype)
+    _load().oracle_h2s(_p(head), _p(out), N, pl.K, Bl, S, Hl * pl.K, D, _esize(head))
+    return out
+
+
+# --------------------------------------------------------------------- attention
+def attn_fwd(Q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float | None = None,
+             causal: bool = True):
+    """Attention from its definition on bf16 bit patterns.
+
+    Q [Bn,S,Hq,D], K,V [Bn,S,Hkv,D] uint16 -> (O [Bn,S,Hq,D] f64, LSE [Bn,Hq,S] f64)."""
+    Q, K, V = (np.ascontiguousarray(a, dtype=np.uint16) for a in (Q, K, V))
+    Bn, S, Hq, D = Q.shape
+    Hkv = K.shape[2]
+    assert K.shape == (Bn, S, Hkv, D) and V.shape == K.shape and Hq % Hkv == 0
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    O = np.empty((Bn, S, Hq, D), dtype=np.float64)
+    LSE = np.empty((Bn, Hq, S), dtype=np.float64)
+    _load().oracle_attn_fwd(_p(Q), _p(K), _p(V), _p(O), _p(LSE), Bn, S, Hq, Hkv, D,
+                            ctypes.c_double(scale), int(causal))
+    return O, LSE
+
+
+def attn_fwd_rows(Q: np.ndarray, K: np.ndarray, V: np.ndarray, rows: np.ndarray,
+                  scale: float | None = None, causal: bool = True):
+    """Selected output rows; ``rows`` is int32 [n,3] of (b, h, i).  Returns
+    (O_rows [n,D] f64, lse_rows [n] f64)."""
+    Q, K, V = (np.ascontiguousarray(a, dtype=np.uint16) for a in (Q, K, V))
+    rows = np.ascontiguousarray(rows, dtype=np.int32).reshape(-1, 3)
+    Bn, S, Hq, D = Q.shape
+    Hkv = K.shape[2]
+    assert K.shape == (Bn, S, Hkv, D) and V.shape == K.shape and Hq % Hkv == 0
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    n = rows.shape[0]
+    O = np.empty((n, D), dtype=np.float64)
+    lse = np.empty((n,), dtype=np.float64)
+    _load().oracle_attn_fwd_rows(_p(Q), _p(K), _p(V), _p(rows), n, _p(O), _p(lse), S, Hq, Hkv,
+                                 D, ctypes.c_double(scale), int(causal))
+    return O, lse
+
+
+# ------------------------------------------------------------------------- layer
+def layer_fwd(Xq: np.ndarray, Xk: np.ndarray, Xv: np.ndarray, pl: Plan,
+              scale: float | None = None, causal: bool = True):
+    """The whole sequence-parallel layer on global tensors, step by step as the
+    paper describes it: partition (Alg. 2) -> all-to-all -> per-rank attention over
+    the rank's head slice -> reverse all-to-all -> collect.
+
+    Xq [B,S,Hq,D], Xk,Xv [B,S,Hkv,D] uint16.  Returns a dict with every intermediate
+    (seq shards, head shards, per-rank O/LSE in fp64) and the global O [B,S,Hq,D]."""
+    qs, ks, vs = partition(Xq, pl), partition(Xk, pl), partition(Xv, pl)
+    qh, kh, vh = s2h(qs, pl), s2h(ks, pl), s2h(vs, pl)
+    N = pl.N
+    oh = np.empty(qh.shape, dtype=np.float64)
+    lse = np.empty((N, pl.Bl, qh.shape[3], pl.S), dtype=np.float64)
+    for r in range(N):
+        oh[r], lse[r] = attn_fwd(qh[r], kh[r], vh[r], scale, causal)
+    os_ = h2s(oh, pl)
+    return dict(q_seq=qs, k_seq=ks, v_seq=vs, q_head=qh, k_head=kh, v_head=vh,
+                o_head=oh, lse_head=lse, o_seq=os_, o_global=gather(os_, pl))
+
+
+# ----------------------------------------------------------------- bf16 helpers
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Exact widening of bf16 bit patterns to fp64."""
+    u = np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << 16
+    return u.view(np.float32).astype(np.float64)

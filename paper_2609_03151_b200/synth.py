@@ -1,0 +1,93 @@
+"""Seeded synthetic inputs shared by the tests, the benchmark and the oracle checks.
+
+Holds none of the method's arithmetic: only the workload table and a random-number
+recipe.  Activations stand in for Llama/Qwen long-context training activations: dense,
+equal-length sequences, i.i.d. N(0,1) drawn in fp32 on GLOBAL coordinates [B,S,H,D] in
+the order Q, K, V (then dO) from one CPU generator, rounded to nearest-even bf16.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    N: int          # virtual ranks
+    B: int          # micro-batch (sequences)
+    S: int          # tokens per sequence
+    Hq: int
+    Hkv: int
+    D: int
+    G: int = 0      # 0 -> BASP (G = B); 1 -> standard Ulysses
+
+    @property
+    def K(self) -> int:
+        return self.N // (self.G or self.B)
+
+    @property
+    def tokens(self) -> int:
+        return self.B * self.S
+
+    def attn_flops_fwd(self) -> float:
+        """4*D flop per unmasked (i,j) pair, S(S+1)/2 pairs per (sequence, q head)."""
+        return 4.0 * self.D * (self.S * (self.S + 1) / 2) * self.B * self.Hq
+
+    def reshard_bytes_s2h(self) -> int:
+        """Q, K and V each read once and written once."""
+        return 2 * 2 * self.B * self.S * (self.Hq + 2 * self.Hkv) * self.D
+
+    def reshard_bytes_h2s(self) -> int:
+        return 2 * 2 * self.B * self.S * self.Hq * self.D
+
+
+WORKLOADS = {
+    "tiny": Workload("tiny", N=4, B=2, S=1024, Hq=8, Hkv=8, D=64),
+    "llama3_8b_32k": Workload("llama3_8b_32k", N=8, B=2, S=32768, Hq=32, Hkv=8, D=128),
+    "sweep_b1": Workload("sweep_b1", N=8, B=1, S=65536, Hq=32, Hkv=8, D=128),
+    "sweep_b2": Workload("sweep_b2", N=8, B=2, S=32768, Hq=32, Hkv=8, D=128),
+    "sweep_b4": Workload("sweep_b4", N=8, B=4, S=16384, Hq=32, Hkv=8, D=128),
+    "sweep_b8": Workload("sweep_b8", N=8, B=8, S=8192, Hq=32, Hkv=8, D=128),
+    "qwen25_7b_64k": Workload("qwen25_7b_64k", N=8, B=2, S=65536, Hq=28, Hkv=4, D=128),
+    "llama3_8b_128k_train": Workload("llama3_8b_128k_train", N=8, B=1, S=131072, Hq=32, Hkv=8, D=128),
+}
+
+
+def shrink(w: Workload, T: int = 512, name: str | None = None) -> Workload:
+    """Same rank/head structure with T tokens per rank (S = T*K)."""
+    return Workload(name or f"{w.name}_T{T}", w.N, w.B, T * w.K, w.Hq, w.Hkv, w.D, w.G)
+
+
+def randn_bf16(gen: torch.Generator, shape) -> torch.Tensor:
+    """N(0,1) in fp32, rounded to nearest-even bf16 (CPU tensor)."""
+    return torch.randn(shape, generator=gen, dtype=torch.float32).to(torch.bfloat16)
+
+
+def make_qkv(w: Workload, seed: int = 0, with_dO: bool = False):
+    """Global Q[B,S,Hq,D], K,V[B,S,Hkv,D] (and dO) as CPU bf16 tensors."""
+    gen = torch.Generator().manual_seed(seed)
+    q = randn_bf16(gen, (w.B, w.S, w.Hq, w.D))
+    k = randn_bf16(gen, (w.B, w.S, w.Hkv, w.D))
+    v = randn_bf16(gen, (w.B, w.S, w.Hkv, w.D))
+    if with_dO:
+        return q, k, v, randn_bf16(gen, (w.B, w.S, w.Hq, w.D))
+    return q, k, v
+
+
+def bits(t: torch.Tensor) -> np.ndarray:
+    """bf16 CPU tensor -> numpy uint16 bit patterns (a copy)."""
+    return t.contiguous().view(torch.int16).numpy().view(np.uint16).copy()
+
+
+def from_bits(a: np.ndarray) -> torch.Tensor:
+    """numpy uint16 bit patterns -> bf16 CPU tensor."""
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.int16).copy()).view(torch.bfloat16)
+
+
+def random_bits(shape, seed: int = 0) -> np.ndarray:
+    """Arbitrary 16-bit patterns (for bit-exact permutation checks)."""
+    rng = np.random.default_rng(seed)
+    return rng.integers(0, 1 << 16, size=shape, dtype=np.uint16)
