@@ -1,0 +1,181 @@
+/*
+ * basp.h -- C ABI of the B200 (sm_100a) BASP attention-layer library (libbasp.so).
+ *
+ * One BASP / Ulysses sequence-parallel attention layer, with the N ranks of the paper
+ * held as N "virtual ranks" whose shards live in ONE GPU's memory:
+ *
+ *   plan            Algorithm 1 (group creation) + Algorithm 2 (sequence partitioning)
+ *   reshard s2h     the group-local all-to-all of Section IV-C, sequence- to head-sharded
+ *   attention       softmax(Q K^T / sqrt(d)) V of Section II-A, causal, per head slice
+ *   reshard h2s     the reverse all-to-all (head- back to sequence-sharded)
+ *   fused layer     the same three steps in one kernel that reads and writes the
+ *                   sequence-sharded shards directly
+ *
+ * Notation: N ranks; B micro-batch (sequences); G groups (G = B is BASP, G = 1 standard
+ * Ulysses); K = N/G ranks per group; Bl = B/G sequences per group; S tokens per sequence;
+ * T = S/K tokens per rank and sequence; Hq / Hkv query / key-value heads; D head dim.
+ *
+ * Shard layouts (dense, row-major, bf16 unless stated):
+ *   sequence-sharded  rank r holds [Bl][T][H][D]    (tokens l*T..(l+1)*T of its sequences)
+ *   head-sharded      rank r holds [Bl][S][H/K][D]  (heads l*H/K..(l+1)*H/K, all tokens)
+ *   LSE               rank r holds fp32 [Bl][Hq/K][S] (natural log of the softmax denominator)
+ * with l = r mod K the local rank and g = r / K the group.
+ *
+ * Conventions for every call
+ *   - returns 0 (BASP_OK) or a negative BASP_ERR_* code; nothing throws across the ABI;
+ *   - "*_shards" arguments are HOST arrays of n_ranks DEVICE pointers; the array is read
+ *     during the call and not retained; every device pointer must be 16-byte aligned;
+ *   - the caller owns every device buffer (workspace included); the library allocates no
+ *     device memory and keeps no pointer after return; the plan is the only library object;
+ *   - launches are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = the
+ *     default stream); no call synchronises the device except basp_get_status and
+ *     basp_layer_fwd_host;
+ *   - there is no CPU fallback: without a CUDA device every launch returns BASP_ERR_CUDA.
+ */
+#ifndef BASP_H_
+#define BASP_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BASP_OK               0
+#define BASP_ERR_INVALID     -1  /* the paper's preconditions fail (N mod G, B > N, S mod K, head splits) */
+#define BASP_ERR_UNSUPPORTED -2  /* valid plan, but outside what the kernels implement               */
+#define BASP_ERR_NULL        -3  /* a required pointer is NULL                                       */
+#define BASP_ERR_ALIGN       -4  /* a device pointer is not 16-byte aligned                          */
+#define BASP_ERR_ALIAS       -5  /* an output shard is also an input shard of an out-of-place step   */
+#define BASP_ERR_CUDA        -6  /* a CUDA call failed; see basp_last_cuda_error                     */
+#define BASP_ERR_TIMEOUT     -7  /* a bounded wait inside a kernel gave up (see basp_get_status)     */
+#define BASP_ERR_WORKSPACE   -8  /* workspace too small                                              */
+
+#define BASP_DTYPE_BF16 0
+#define BASP_MAX_RANKS  32
+
+typedef struct basp_plan basp_plan; /* opaque; host memory; immutable; may be shared by threads */
+
+/* Algorithm 1's inputs (world size N, micro-batch B) plus the tensor shape of the layer. */
+typedef struct basp_config {
+    int n_ranks;     /* N, 1..BASP_MAX_RANKS                                              */
+    int micro_batch; /* B                                                                 */
+    int num_groups;  /* G: 0 -> B (BASP, Algorithm 1); 1 -> standard Ulysses; must divide N and B */
+    int seq_len;     /* S, tokens per sequence                                            */
+    int n_q_heads;   /* Hq                                                                */
+    int n_kv_heads;  /* Hkv (Hq mod Hkv = 0; query head h reads KV head h / (Hq/Hkv))     */
+    int head_dim;    /* D                                                                 */
+    int dtype;       /* BASP_DTYPE_BF16                                                   */
+    int causal;      /* 1: key j visible to query i iff j <= i; 0: full attention         */
+} basp_config;
+
+typedef struct basp_plan_info {
+    int group_size;        /* K = N / G  (all-to-all participants; Table I)               */
+    int num_groups;        /* G                                                           */
+    int seqs_per_group;    /* Bl = B / G                                                  */
+    int tokens_per_rank;   /* T = S / K  (per sequence; tokens per rank = Bl * T = B*S/N) */
+    int q_heads_per_rank;  /* Hq / K                                                      */
+    int kv_heads_per_rank; /* Hkv / K                                                     */
+    size_t q_shard_elems;  /* elements of one rank's Q (or O) shard, either layout        */
+    size_t kv_shard_elems; /* elements of one rank's K (or V) shard, either layout        */
+    size_t lse_shard_elems;/* fp32 elements of one rank's LSE                             */
+} basp_plan_info;
+
+/* Algorithm 2's outputs for one rank. Ranges are half-open. */
+typedef struct basp_rank_info {
+    int group, local_rank;
+    int seq_begin, seq_end;         /* sequences of the micro-batch this rank works on     */
+    int token_begin, token_end;     /* its token range inside each of those sequences      */
+    int q_head_begin, q_head_end;   /* heads it owns after the first all-to-all            */
+    int kv_head_begin, kv_head_end;
+} basp_rank_info;
+
+/* ---- plan: Algorithm 1 (K = N/B, contiguous rank blocks, N mod B = 0 asserted) and
+ * Algorithm 2 (group = r / K, local = r mod K, chunk = S / K), generalised to G groups
+ * as in the workload-equivalence paragraph of Section IV-C.
+ * Errors: BASP_ERR_NULL; BASP_ERR_INVALID for N mod G != 0, B mod G != 0, B > N in BASP
+ * mode (the paper's data-parallel fallback is not provided), S mod K != 0, Hq mod Hkv != 0,
+ * Hq mod K != 0, Hkv mod K != 0; BASP_ERR_UNSUPPORTED for dtype != bf16, N > BASP_MAX_RANKS
+ * or a head slice whose row ((H/K)*D*2 bytes) is not a multiple of 16 bytes.
+ * On success *out owns a host object; release it with basp_plan_destroy. */
+int basp_plan_create(const basp_config *cfg, basp_plan **out);
+int basp_plan_destroy(basp_plan *plan);
+int basp_plan_get_info(const basp_plan *plan, basp_plan_info *info);
+int basp_plan_get_rank(const basp_plan *plan, int rank, basp_rank_info *info);
+/* ranks_out: host array of K ints; group i is ranks i*K .. i*K+K-1 (Algorithm 1). */
+int basp_plan_group_ranks(const basp_plan *plan, int group, int *ranks_out);
+
+/* ---- reshards: the two all-to-alls of the Ulysses layer confined to each group
+ * (Section II-C, Section IV-C), as out-of-place permutations inside device memory.
+ *   s2h: head[gK+m][bl][s][h'][d] = seq[gK + s/T][bl][s mod T][m*H/K + h'][d]
+ *   h2s: seq[gK+l][bl][t][m*H/K + h'][d] = head[gK+m][bl][l*T + t][h'][d]
+ * n_heads = H must be a multiple of K with (H/K)*D*2 bytes a multiple of 16.  Bit-exact.
+ * Errors: NULL / ALIGN / ALIAS (a destination shard equal to a source shard) / INVALID
+ * (n_heads) / CUDA. */
+int basp_reshard_s2h(const basp_plan *plan, int n_heads, const void *const *seq_shards,
+                     void *const *head_shards, void *stream);
+int basp_reshard_h2s(const basp_plan *plan, int n_heads, const void *const *head_shards,
+                     void *const *seq_shards, void *stream);
+/* Q (Hq heads), K and V (Hkv heads) in ONE launch. */
+int basp_reshard_qkv_s2h(const basp_plan *plan, const void *const *q_seq, const void *const *k_seq,
+                         const void *const *v_seq, void *const *q_head, void *const *k_head,
+                         void *const *v_head, void *stream);
+
+/* ---- attention over each rank's head slice (Section II-A equation; the tiled,
+ * online-softmax evaluation the paper cites from FlashAttention):
+ *   O[i] = sum_{j visible} softmax_j(scale * q_i . k_j) v_j,   LSE[i] = ln sum_j exp(scale * q_i . k_j)
+ * Inputs/outputs are HEAD-sharded; lse_shards may be NULL (then no LSE is written), else a
+ * host array of n_ranks device pointers to fp32 [Bl][Hq/K][S].  softmax_scale = 0 selects
+ * 1/sqrt(D).  bf16 operands, fp32 accumulation and softmax, P rounded to bf16 before P.V.
+ * Requires D in {64, 128} and S a multiple of 128 (else BASP_ERR_UNSUPPORTED).
+ * A bounded wait that expires inside the kernel is reported by basp_get_status. */
+int basp_attn_fwd(const basp_plan *plan, const void *const *q_head, const void *const *k_head,
+                  const void *const *v_head, void *const *o_head, float *const *lse_shards,
+                  float softmax_scale, void *stream);
+
+/* ---- the whole layer on SEQUENCE-sharded shards: s2h(Q,K,V) -> attention -> h2s(O).
+ * `workspace` is device memory of at least basp_workspace_bytes(plan) bytes (16-byte
+ * aligned) that receives the head-sharded Q, K, V and O; its contents afterwards are
+ * unspecified.  Three launches.  Errors as above plus BASP_ERR_WORKSPACE. */
+int basp_layer_fwd(const basp_plan *plan, const void *const *q_seq, const void *const *k_seq,
+                   const void *const *v_seq, void *const *o_seq, float *const *lse_shards,
+                   void *workspace, size_t workspace_bytes, float softmax_scale, void *stream);
+size_t basp_workspace_bytes(const basp_plan *plan);
+
+/* ---- the same layer as ONE kernel: attention tiles are fetched straight from the
+ * sequence-sharded sources (token tile at sequence position s lives on rank gK + s/T) and
+ * O tiles are stored straight into the sequence-sharded destination, so the head-sharded
+ * copies never exist.  Additionally requires T to be a multiple of 128.  No workspace. */
+int basp_layer_fwd_fused(const basp_plan *plan, const void *const *q_seq, const void *const *k_seq,
+                         const void *const *v_seq, void *const *o_seq, float *const *lse_shards,
+                         float softmax_scale, void *stream);
+
+/* ---- the fused layer for callers whose shards are in HOST memory: copies every Q/K/V
+ * shard host->device into `device_arena` (device memory, >= basp_host_arena_bytes(plan)
+ * bytes), runs basp_layer_fwd_fused, copies every O shard device->host and waits for the
+ * stream.  q/k/v/o_seq_host are host arrays of n_ranks HOST pointers (pinned memory makes
+ * the copies asynchronous; pageable memory works, slower). */
+int basp_layer_fwd_host(const basp_plan *plan, const void *const *q_seq_host,
+                        const void *const *k_seq_host, const void *const *v_seq_host,
+                        void *const *o_seq_host, void *device_arena, size_t arena_bytes,
+                        float softmax_scale, void *stream);
+size_t basp_host_arena_bytes(const basp_plan *plan);
+
+/* ---- device status.  Every wait inside the kernels (on a shared-memory barrier) is bounded;
+ * when one expires the kernel records where, lets its copies drain, frees its tensor memory
+ * and returns.  basp_get_status synchronises `stream`, copies the four status words of the
+ * current device to status_out (host, 4 ints: {code, role, block, detail}; may be NULL) and
+ * returns BASP_OK or BASP_ERR_TIMEOUT.  basp_clear_status zeroes them (asynchronously). */
+int basp_get_status(void *stream, int *status_out);
+int basp_clear_status(void *stream);
+
+const char *basp_strerror(int code);
+/* Text of the last CUDA error seen by the calling thread inside this library ("" if none). */
+const char *basp_last_cuda_error(void);
+/* Number of kernel launches issued by this library in the calling process so far. */
+long long basp_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BASP_H_ */

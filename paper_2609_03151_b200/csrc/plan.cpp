@@ -1,0 +1,78 @@
+// Group planner: Algorithm 1 (batch-aware group creation) and Algorithm 2 (batch-aware
+// sequence partitioning) as integer arithmetic on the host.  No communicator is built:
+// a group is the contiguous rank range [g*K, (g+1)*K).
+#include <new>
+
+#include "plan.h"
+
+extern "C" int basp_plan_create(const basp_config *cfg, basp_plan **out) {
+    if (!cfg || !out) return BASP_ERR_NULL;
+    *out = nullptr;
+    const int N = cfg->n_ranks, B = cfg->micro_batch, S = cfg->seq_len;
+    const int Hq = cfg->n_q_heads, Hkv = cfg->n_kv_heads, D = cfg->head_dim;
+    if (N <= 0 || B <= 0 || S <= 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || cfg->num_groups < 0)
+        return BASP_ERR_INVALID;
+    const int G = cfg->num_groups == 0 ? B : cfg->num_groups;   // Algorithm 1: num_groups = B
+    if (G == B && B > N) return BASP_ERR_INVALID;               // data-parallel fallback: not a plan
+    if (N % G != 0 || B % G != 0) return BASP_ERR_INVALID;      // Algorithm 1: assert N mod B = 0
+    const int K = N / G;                                         // Algorithm 1: K = N / B
+    if (S % K != 0) return BASP_ERR_INVALID;                     // Algorithm 2: chunk = L / K
+    if (Hq % Hkv != 0 || Hq % K != 0 || Hkv % K != 0) return BASP_ERR_INVALID;
+    if (cfg->dtype != BASP_DTYPE_BF16 || N > BASP_MAX_RANKS) return BASP_ERR_UNSUPPORTED;
+    if (((Hkv / K) * D * 2) % 16 != 0 || ((Hq / K) * D * 2) % 16 != 0) return BASP_ERR_UNSUPPORTED;
+    if (cfg->causal != 0 && cfg->causal != 1) return BASP_ERR_INVALID;
+
+    basp_plan *p = new (std::nothrow) basp_plan;
+    if (!p) return BASP_ERR_INVALID;
+    p->cfg = *cfg;
+    p->N = N; p->B = B; p->G = G; p->K = K; p->Bl = B / G; p->S = S; p->T = S / K;
+    p->Hq = Hq; p->Hkv = Hkv; p->D = D; p->Hq_l = Hq / K; p->Hkv_l = Hkv / K;
+    p->causal = cfg->causal;
+    *out = p;
+    return BASP_OK;
+}
+
+extern "C" int basp_plan_destroy(basp_plan *plan) {
+    if (!plan) return BASP_ERR_NULL;
+    delete plan;
+    return BASP_OK;
+}
+
+extern "C" int basp_plan_get_info(const basp_plan *p, basp_plan_info *info) {
+    if (!p || !info) return BASP_ERR_NULL;
+    info->group_size = p->K;
+    info->num_groups = p->G;
+    info->seqs_per_group = p->Bl;
+    info->tokens_per_rank = p->T;
+    info->q_heads_per_rank = p->Hq_l;
+    info->kv_heads_per_rank = p->Hkv_l;
+    // Workload equivalence (Section IV-C): Bl*T*H*D = (B*S/N)*H*D for every grouping.
+    info->q_shard_elems = (size_t)p->Bl * p->T * p->Hq * p->D;
+    info->kv_shard_elems = (size_t)p->Bl * p->T * p->Hkv * p->D;
+    info->lse_shard_elems = (size_t)p->Bl * p->Hq_l * p->S;
+    return BASP_OK;
+}
+
+extern "C" int basp_plan_get_rank(const basp_plan *p, int r, basp_rank_info *info) {
+    if (!p || !info) return BASP_ERR_NULL;
+    if (r < 0 || r >= p->N) return BASP_ERR_INVALID;
+    const int g = r / p->K, l = r % p->K;       // Algorithm 2: my_group, my_local_rank
+    info->group = g;
+    info->local_rank = l;
+    info->seq_begin = g * p->Bl;                // Algorithm 2: seq_start = my_group (Bl = 1)
+    info->seq_end = (g + 1) * p->Bl;
+    info->token_begin = l * p->T;               // Algorithm 2: token_start = local * chunk
+    info->token_end = (l + 1) * p->T;
+    info->q_head_begin = l * p->Hq_l;
+    info->q_head_end = (l + 1) * p->Hq_l;
+    info->kv_head_begin = l * p->Hkv_l;
+    info->kv_head_end = (l + 1) * p->Hkv_l;
+    return BASP_OK;
+}
+
+extern "C" int basp_plan_group_ranks(const basp_plan *p, int group, int *ranks_out) {
+    if (!p || !ranks_out) return BASP_ERR_NULL;
+    if (group < 0 || group >= p->G) return BASP_ERR_INVALID;
+    for (int j = 0; j < p->K; ++j) ranks_out[j] = group * p->K + j;   // Algorithm 1: [iK .. iK+K-1]
+    return BASP_OK;
+}

@@ -1,0 +1,175 @@
+// Group-local all-to-alls of the Ulysses layer (Section II-C, Section IV-C) as in-HBM
+// permutations between N virtual ranks.
+//
+//   s2h: head[gK+m][bl][s][h'][d] = seq[gK + s/T][bl][s mod T][m*H/K + h'][d]
+//   h2s: the inverse map.
+//
+// The unit moved is a 16-byte vector.  Walking the SEQUENCE-sharded side in memory order, a
+// token row of H*D elements is K consecutive runs of (H/K)*D elements, run m belonging to
+// local rank m of the group; on the head-sharded side each run is contiguous too.  So both
+// sides are touched in runs of >= 256 bytes and every 128-byte line is moved whole.  One
+// launch covers up to three tensors (Q, K, V) of all ranks.
+//
+// HBM-bound: 2 bytes of traffic per byte of tensor, no arithmetic.  Each thread keeps U
+// independent 16-byte streaming loads in flight before its stores.
+#include "common.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kUnroll = 8;                       // vectors per thread and chunk
+constexpr uint32_t kChunkV = kThreads * kUnroll; // 32 KiB per CTA
+
+struct ReshardTensor {
+    const char *seq[BASP_MAX_RANKS];
+    const char *head[BASP_MAX_RANKS];
+    uint32_t row_v;            // vectors per token row on the sequence-sharded side (K runs)
+    uint32_t run_v;            // vectors per run = (H/K)*D*2/16
+    uint32_t shard_v;          // vectors per rank shard
+    uint32_t chunks_per_shard;
+    uint32_t chunk_begin;      // first CTA index of this tensor
+    FastDiv div_row, div_run;
+};
+
+struct ReshardParams {
+    int n_tensors;
+    uint32_t K, T, S;
+    FastDiv div_T;
+    ReshardTensor t[3];
+};
+
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
+    uint4 v;
+    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream(uint4 *p, const uint4 &v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// kToHead = true: s2h (read the sequence side in order, scatter runs to the head side);
+// false: h2s (gather runs from the head side, write the sequence side in order).
+template <bool kToHead>
+__global__ void __launch_bounds__(kThreads) reshard_kernel(const __grid_constant__ ReshardParams p) {
+    uint32_t c = blockIdx.x;
+    int ti = 0;
+    while (ti + 1 < p.n_tensors && c >= p.t[ti + 1].chunk_begin) ++ti;
+    const ReshardTensor &t = p.t[ti];
+    c -= t.chunk_begin;
+    const uint32_t r = c / t.chunks_per_shard;
+    const uint32_t chunk = c - r * t.chunks_per_shard;
+    const uint32_t g = r / p.K, l = r - g * p.K;
+    const uint32_t v0 = chunk * kChunkV + threadIdx.x;
+
+    const uint4 *seq = reinterpret_cast<const uint4 *>(t.seq[r]);
+    const uint4 *hp[kUnroll];   // address on the head-sharded side of each vector
+#pragma unroll
+    for (int i = 0; i < kUnroll; ++i) {
+        const uint32_t v = v0 + i * kThreads;
+        const uint32_t vv = v < t.shard_v ? v : 0;
+        const uint32_t tok = fdiv(vv, t.div_row);          // (bl, t) flattened
+        const uint32_t col = vv - tok * t.row_v;
+        const uint32_t m = fdiv(col, t.div_run);           // destination local rank
+        const uint32_t j = col - m * t.run_v;
+        const uint32_t bl = fdiv(tok, p.div_T);
+        const uint32_t tt = tok - bl * p.T;
+        const uint32_t hv = (bl * p.S + l * p.T + tt) * t.run_v + j;
+        hp[i] = reinterpret_cast<const uint4 *>(t.head[g * p.K + m]) + hv;
+    }
+    uint4 data[kUnroll];
+#pragma unroll
+    for (int i = 0; i < kUnroll; ++i) {
+        const uint32_t v = v0 + i * kThreads;
+        if (v < t.shard_v) data[i] = ld_stream(kToHead ? seq + v : hp[i]);
+    }
+#pragma unroll
+    for (int i = 0; i < kUnroll; ++i) {
+        const uint32_t v = v0 + i * kThreads;
+        if (v < t.shard_v) st_stream(const_cast<uint4 *>(kToHead ? hp[i] : seq + v), data[i]);
+    }
+}
+
+struct TensorArg {
+    int n_heads;
+    const void *const *seq;
+    const void *const *head;
+};
+
+int fill_tensor(const basp_plan *p, const TensorArg &a, bool to_head, ReshardTensor *t, uint32_t *chunk_cursor) {
+    if (!a.seq || !a.head) return BASP_ERR_NULL;
+    if (a.n_heads <= 0 || a.n_heads % p->K != 0) return BASP_ERR_INVALID;
+    const size_t run_bytes = (size_t)(a.n_heads / p->K) * p->D * 2;
+    if (run_bytes % 16 != 0) return BASP_ERR_UNSUPPORTED;
+    const size_t shard_bytes = (size_t)p->Bl * p->T * a.n_heads * p->D * 2;
+    if (shard_bytes / 16 >= (1ull << 31)) return BASP_ERR_UNSUPPORTED;
+    for (int r = 0; r < p->N; ++r) {
+        if (!a.seq[r] || !a.head[r]) return BASP_ERR_NULL;
+        if (!aligned16(a.seq[r]) || !aligned16(a.head[r])) return BASP_ERR_ALIGN;
+        t->seq[r] = (const char *)a.seq[r];
+        t->head[r] = (const char *)a.head[r];
+    }
+    // out-of-place only: no destination shard may overlap a source shard
+    const void *const *src = to_head ? a.seq : a.head;
+    const void *const *dst = to_head ? a.head : a.seq;
+    for (int i = 0; i < p->N; ++i)
+        for (int j = 0; j < p->N; ++j) {
+            const char *s = (const char *)src[i], *d = (const char *)dst[j];
+            if (s < d + shard_bytes && d < s + shard_bytes) return BASP_ERR_ALIAS;
+        }
+    t->run_v = (uint32_t)(run_bytes / 16);
+    t->row_v = t->run_v * p->K;
+    t->shard_v = (uint32_t)(shard_bytes / 16);
+    t->chunks_per_shard = (t->shard_v + kChunkV - 1) / kChunkV;
+    t->chunk_begin = *chunk_cursor;
+    t->div_row = make_fastdiv(t->row_v);
+    t->div_run = make_fastdiv(t->run_v);
+    *chunk_cursor += t->chunks_per_shard * (uint32_t)p->N;
+    return BASP_OK;
+}
+
+int launch(const basp_plan *p, const TensorArg *args, int n, bool to_head, void *stream) {
+    if (!p) return BASP_ERR_NULL;
+    ReshardParams prm;
+    prm.n_tensors = n;
+    prm.K = p->K; prm.T = p->T; prm.S = p->S;
+    prm.div_T = make_fastdiv((uint32_t)p->T);
+    uint32_t chunks = 0;
+    for (int i = 0; i < n; ++i) {
+        int rc = fill_tensor(p, args[i], to_head, &prm.t[i], &chunks);
+        if (rc != BASP_OK) return rc;
+    }
+    if (chunks == 0) return BASP_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (to_head) reshard_kernel<true><<<chunks, kThreads, 0, st>>>(prm);
+    else         reshard_kernel<false><<<chunks, kThreads, 0, st>>>(prm);
+    BASP_CUDA_TRY(cudaGetLastError());
+    basp_count_launch(1);
+    return BASP_OK;
+}
+
+}  // namespace
+
+extern "C" int basp_reshard_s2h(const basp_plan *plan, int n_heads, const void *const *seq_shards,
+                                void *const *head_shards, void *stream) {
+    TensorArg a{n_heads, seq_shards, (const void *const *)head_shards};
+    return launch(plan, &a, 1, true, stream);
+}
+
+extern "C" int basp_reshard_h2s(const basp_plan *plan, int n_heads, const void *const *head_shards,
+                                void *const *seq_shards, void *stream) {
+    TensorArg a{n_heads, (const void *const *)seq_shards, head_shards};
+    return launch(plan, &a, 1, false, stream);
+}
+
+extern "C" int basp_reshard_qkv_s2h(const basp_plan *plan, const void *const *q_seq,
+                                    const void *const *k_seq, const void *const *v_seq,
+                                    void *const *q_head, void *const *k_head, void *const *v_head,
+                                    void *stream) {
+    if (!plan) return BASP_ERR_NULL;
+    TensorArg a[3] = {{plan->Hq, q_seq, (const void *const *)q_head},
+                      {plan->Hkv, k_seq, (const void *const *)k_head},
+                      {plan->Hkv, v_seq, (const void *const *)v_head}};
+    return launch(plan, a, 3, true, stream);
+}

@@ -1,0 +1,106 @@
+"""The whole layer through the C ABI: three-launch path and fused kernel against the oracle's
+layer, BASP = Ulysses = unpartitioned on the GPU, the host-buffer entry, and full-size sampled parity."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import assert_attn_close, make_plan, oracle_inputs, to_dev, to_f64
+from paper_2609_03151_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def gpu_layer(basp, w, Xq, Xk, Xv, op, fused):
+    pl = make_plan(basp, w)
+    dq, dk, dv = (to_dev(oracle.partition(X, op)) for X in (Xq, Xk, Xv))
+    do = [torch.zeros_like(t) for t in dq]
+    basp.basp_clear_status()
+    if fused:
+        basp.basp_layer_fwd_fused(pl, dq, dk, dv, do)
+    else:
+        ws = torch.empty(basp.basp_workspace_bytes(pl), dtype=torch.uint8, device="cuda")
+        basp.basp_layer_fwd(pl, dq, dk, dv, do, ws)
+    basp.basp_get_status()
+    return do
+
+
+@pytest.mark.parametrize("fused", [False, True])
+@pytest.mark.parametrize("w", [
+    synth.WORKLOADS["tiny"],
+    synth.shrink(synth.WORKLOADS["llama3_8b_32k"], 256),
+    synth.shrink(synth.WORKLOADS["sweep_b1"], 128),
+    synth.shrink(synth.WORKLOADS["sweep_b8"], 256),
+    synth.shrink(synth.WORKLOADS["qwen25_7b_64k"], 128),
+], ids=lambda w: w.name)
+def test_layer_matches_oracle(basp, w, fused):
+    Xq, Xk, Xv, op = oracle_inputs(w)
+    ref = oracle.layer_fwd(Xq, Xk, Xv, op)
+    do = gpu_layer(basp, w, Xq, Xk, Xv, op, fused)
+    assert_attn_close(to_f64(do), ref["o_seq"], f"{w.name} fused={fused}")
+
+
+def test_tiny_basp_equals_ulysses_equals_unpartitioned(basp):
+    """BASELINE config 1: b=2 (two groups of 2) vs b-agnostic Ulysses (one group of 4) vs no partition.
+    The per-row tile schedule does not depend on the grouping, so the GPU outputs agree bit for bit."""
+    w = synth.WORKLOADS["tiny"]
+    Xq, Xk, Xv, op = oracle_inputs(w)
+    full, _ = oracle.attn_fwd(Xq, Xk, Xv)
+    outs = {}
+    for name, ww in (("basp", w), ("ulysses", synth.Workload("u", 4, 2, 1024, 8, 8, 64, G=1)),
+                     ("single", synth.Workload("s", 2, 2, 1024, 8, 8, 64))):
+        o = oracle.plan(ww.N, ww.B, ww.S, ww.G)
+        for fused in (False, True):
+            do = gpu_layer(basp, ww, Xq, Xk, Xv, o, fused)
+            bits = np.stack([synth.bits(t.cpu()) for t in do])
+            outs[(name, fused)] = oracle.gather(bits, o)
+            assert_attn_close(oracle.bf16_bits_to_f64(outs[(name, fused)]), full, f"{name} fused={fused}")
+    first = outs[("basp", False)]
+    for key, val in outs.items():
+        assert np.array_equal(val, first), key
+
+
+def test_host_buffer_entry(basp):
+    w = synth.shrink(synth.WORKLOADS["llama3_8b_32k"], 128)
+    Xq, Xk, Xv, op = oracle_inputs(w, seed=2)
+    ref = oracle.layer_fwd(Xq, Xk, Xv, op)
+    pl = make_plan(basp, w)
+    host = [[synth.from_bits(a[r]).pin_memory() for r in range(w.N)] for a in (ref["q_seq"], ref["k_seq"], ref["v_seq"])]
+    out = [torch.zeros_like(t).pin_memory() for t in host[0]]
+    arena = torch.empty(basp.basp_host_arena_bytes(pl), dtype=torch.uint8, device="cuda")
+    basp.basp_clear_status()
+    basp.basp_layer_fwd_host(pl, host[0], host[1], host[2], out, arena)
+    basp.basp_get_status()
+    assert_attn_close(to_f64(out), ref["o_seq"], "host entry")
+
+
+@pytest.mark.parametrize("name", ["llama3_8b_32k"])
+def test_full_size_sampled_rows(basp, name):
+    """BASELINE config 2 at full size, the launches the benchmark times: sampled output rows
+    (first rows, shard and tile boundaries, last rows, random rows) against oracle rows."""
+    w = synth.WORKLOADS[name]
+    q, k, v = synth.make_qkv(w, seed=0)
+    pl = make_plan(basp, w)
+    T, K = pl.T, pl.K
+
+    def shards(x):   # Algorithm 2 by slicing
+        return [x[r // K: r // K + 1, (r % K) * T:(r % K + 1) * T].contiguous().cuda() for r in range(w.N)]
+
+    dq, dk, dv = shards(q), shards(k), shards(v)
+    rng = np.random.default_rng(0)
+    cand = [0, 1, 127, 128, 255, 256, T - 1, T, T + 1, 2 * T - 1, 2 * T, w.S - 129, w.S - 128, w.S - 1]
+    rows = [(b, h, i) for b in range(w.B) for h in (0, 5, w.Hq - 1) for i in cand]
+    rows += [(int(rng.integers(w.B)), int(rng.integers(w.Hq)), int(rng.integers(w.S))) for _ in range(40)]
+    rows = np.array(rows, dtype=np.int32)
+    ref, _ = oracle.attn_fwd_rows(synth.bits(q), synth.bits(k), synth.bits(v), rows)
+    ws = torch.empty(basp.basp_workspace_bytes(pl), dtype=torch.uint8, device="cuda")
+    for fused in (False, True):
+        do = [torch.zeros_like(t) for t in dq]
+        basp.basp_clear_status()
+        if fused:
+            basp.basp_layer_fwd_fused(pl, dq, dk, dv, do)
+        else:
+            basp.basp_layer_fwd(pl, dq, dk, dv, do, ws)
+        basp.basp_get_status()
+        got = np.stack([do[b * K + i // T][0, i % T, h].float().cpu().numpy().astype(np.float64) for b, h, i in rows])
+        assert_attn_close(got, ref, f"{name} fused={fused}")

@@ -1,0 +1,80 @@
+"""CPU-only checks of the C ABI: every declared symbol is exported, the host planner agrees
+with the oracle's Algorithm 1 / Algorithm 2, and the argument checks that need no GPU."""
+import os
+import re
+
+import pytest
+
+import oracle
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_every_declared_symbol_is_exported(basp):
+    text = open(os.path.join(ROOT, "include", "basp.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = set(re.findall(r"\b(basp_[a-z0-9_]+)\s*\(", text))
+    assert declared == set(basp.EXPORTS), declared ^ set(basp.EXPORTS)
+    for name in declared:
+        assert hasattr(basp.lib, name), name
+
+
+@pytest.mark.parametrize("N,B,G", [(4, 2, 0), (8, 1, 0), (8, 2, 0), (8, 4, 0), (8, 8, 0), (8, 4, 1), (8, 4, 2), (16, 4, 0)])
+def test_plan_matches_oracle(basp, N, B, G):
+    S, Hq, Hkv, D = 4096, 32, 16, 128
+    pl = basp.basp_plan_create(N, B, S, Hq, Hkv, D, num_groups=G)
+    op = oracle.plan(N, B, S, G)
+    assert (pl.K, pl.G, pl.Bl, pl.T) == (op.K, op.G, op.Bl, op.T)
+    assert pl.info.q_shard_elems == B * S // N * Hq * D          # tokens per GPU = B*S/N (Table I)
+    assert pl.info.kv_shard_elems == B * S // N * Hkv * D
+    for g in range(pl.G):
+        assert basp.basp_plan_group_ranks(pl, g) == op.group_ranks(g)
+    for r in range(N):
+        assert basp.basp_plan_get_rank(pl, r) == op.rank_info(r, Hq, Hkv)
+
+
+def test_paper_example_four_gpus_batch_two(basp):
+    pl = basp.basp_plan_create(4, 2, 1024, 8, 8, 64)
+    assert pl.K == 2 and [basp.basp_plan_group_ranks(pl, g) for g in range(2)] == [[0, 1], [2, 3]]
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(n_ranks=8, micro_batch=3), -1),                 # N mod B != 0
+    (dict(n_ranks=4, micro_batch=8), -1),                 # B > N
+    (dict(seq_len=1022), -1),                             # S mod K != 0
+    (dict(n_q_heads=30), -1),                             # Hq mod Hkv
+    (dict(n_kv_heads=2), -1),                             # Hkv mod K (K = 4)
+    (dict(num_groups=3), -1),
+    (dict(dtype=1), -2),
+    (dict(n_ranks=64, micro_batch=64), -2),               # more than BASP_MAX_RANKS
+    (dict(head_dim=3, n_q_heads=4, n_kv_heads=4), -2),    # rows not a multiple of 16 bytes
+])
+def test_plan_errors(basp, kw, code):
+    args = dict(n_ranks=8, micro_batch=2, seq_len=1024, n_q_heads=32, n_kv_heads=8, head_dim=128)
+    args.update(kw)
+    with pytest.raises(basp.BaspError) as e:
+        basp.basp_plan_create(**args)
+    assert e.value.code == code
+
+
+def test_null_and_alignment_checks_need_no_gpu(basp):
+    import ctypes
+    pl = basp.basp_plan_create(4, 2, 1024, 8, 8, 64)
+    n = 4
+    good = (ctypes.c_void_p * n)(*[0x10000 * (i + 1) for i in range(n)])
+    good2 = (ctypes.c_void_p * n)(*[0x10000000 + 0x100000 * (i + 1) for i in range(n)])
+    odd = (ctypes.c_void_p * n)(*[0x10000 * (i + 1) + 8 for i in range(n)])
+    null = (ctypes.c_void_p * n)(*[None] * n)
+    L = basp.lib
+    assert L.basp_reshard_s2h(pl.handle, 8, None, good, None) == basp.BASP_ERR_NULL
+    assert L.basp_reshard_s2h(pl.handle, 8, null, good, None) == basp.BASP_ERR_NULL
+    assert L.basp_reshard_s2h(pl.handle, 8, odd, good2, None) == basp.BASP_ERR_ALIGN
+    assert L.basp_reshard_s2h(pl.handle, 8, good, good, None) == basp.BASP_ERR_ALIAS
+    assert L.basp_reshard_s2h(pl.handle, 7, good, good2, None) == basp.BASP_ERR_INVALID
+    assert L.basp_attn_fwd(pl.handle, good, good, good, None, None, 0.0, None) == basp.BASP_ERR_NULL
+    assert L.basp_attn_fwd(pl.handle, good, good, good, good, None, 0.0, None) == basp.BASP_ERR_ALIAS
+    assert L.basp_layer_fwd(pl.handle, good, good, good, good2, None, ctypes.c_void_p(0x1000), 16, 0.0, None) \
+        == basp.BASP_ERR_WORKSPACE
+    pl2 = basp.basp_plan_create(4, 2, 1000, 8, 8, 64)    # S not a multiple of 128
+    assert L.basp_attn_fwd(pl2.handle, good, good, good, good2, None, 0.0, None) == basp.BASP_ERR_UNSUPPORTED
+    assert basp.lib.basp_strerror(-7).decode().startswith("a bounded wait")
