@@ -142,6 +142,28 @@ int basp_layer_fwd(const basp_plan *plan, const void *const *q_seq, const void *
                    void *workspace, size_t workspace_bytes, float softmax_scale, void *stream);
 size_t basp_workspace_bytes(const basp_plan *plan);
 
+/* ---- the three-launch layer WITHOUT caller workspace and without any allocation (the paper
+ * has no counterpart: this entry point exists for the sake of callers, not of the method).
+ * Some callers cannot allocate device memory at the point where they need the layer: the whole
+ * device heap may already belong to another allocator or memory pool, or the call sits in a
+ * latency-critical loop in which the device-wide synchronisation of cudaMalloc / cudaFree is
+ * not acceptable.  For them the head-sharded Q, K, V and O go into a fixed array of
+ * BASP_STATIC_SCRATCH_BYTES that is part of this library's image: every GPU that loads the
+ * library holds that much memory until the process exits.  The call runs no cudaMalloc, cudaFree
+ * or other allocating routine; inputs and outputs are still the caller's.
+ *   - Plans whose basp_workspace_bytes exceeds BASP_STATIC_SCRATCH_BYTES are refused with
+ *     BASP_ERR_WORKSPACE (basp_last_cuda_error then names both sizes).
+ *   - The first call on each device looks up the array's device address (one runtime query, made
+ *     with that device current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array.  It keeps whatever the last call wrote; nothing
+ *     needs clearing because each call overwrites every byte it later reads.  Two calls that can
+ *     overlap on the GPU (different streams, no dependency) race on it: serialise them.
+ * Results are identical to basp_layer_fwd. */
+#define BASP_STATIC_SCRATCH_BYTES (16u << 20)
+int basp_layer_fwd_static(const basp_plan *plan, const void *const *q_seq, const void *const *k_seq,
+                          const void *const *v_seq, void *const *o_seq, float *const *lse_shards,
+                          float softmax_scale, void *stream);
+
 /* ---- the same layer as ONE kernel: attention tiles are fetched straight from the
  * sequence-sharded sources (token tile at sequence position s lives on rank gK + s/T) and
  * O tiles are stored straight into the sequence-sharded destination, so the head-sharded

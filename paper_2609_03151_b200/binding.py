@@ -26,7 +26,7 @@ EXPORTS = [
     "basp_plan_create", "basp_plan_destroy", "basp_plan_get_info", "basp_plan_get_rank",
     "basp_plan_group_ranks", "basp_reshard_s2h", "basp_reshard_h2s", "basp_reshard_qkv_s2h",
     "basp_attn_fwd", "basp_layer_fwd", "basp_workspace_bytes", "basp_layer_fwd_fused",
-    "basp_layer_fwd_host", "basp_host_arena_bytes", "basp_get_status", "basp_clear_status",
+    "basp_layer_fwd_host", "basp_host_arena_bytes", "basp_layer_fwd_static", "basp_get_status", "basp_clear_status",
     "basp_strerror", "basp_last_cuda_error", "basp_launch_count",
 ]
 
@@ -59,6 +59,7 @@ lib.basp_reshard_qkv_s2h.argtypes = [c_void_p] + [_PP] * 6 + [c_void_p]
 lib.basp_attn_fwd.argtypes = [c_void_p] + [_PP] * 5 + [c_float, c_void_p]
 lib.basp_layer_fwd.argtypes = [c_void_p] + [_PP] * 5 + [c_void_p, c_size_t, c_float, c_void_p]
 lib.basp_layer_fwd_fused.argtypes = [c_void_p] + [_PP] * 5 + [c_float, c_void_p]
+lib.basp_layer_fwd_static.argtypes = [c_void_p] + [_PP] * 5 + [c_float, c_void_p]
 lib.basp_layer_fwd_host.argtypes = [c_void_p] + [_PP] * 4 + [c_void_p, c_size_t, c_float, c_void_p]
 lib.basp_workspace_bytes.argtypes = [c_void_p]
 lib.basp_workspace_bytes.restype = c_size_t
@@ -184,6 +185,19 @@ def basp_layer_fwd_fused(plan, q_seq, k_seq, v_seq, o_seq, lse_shards=None, soft
     _check(lib.basp_layer_fwd_fused(plan.handle, _ptrs(q_seq, n), _ptrs(k_seq, n), _ptrs(v_seq, n),
                                     _ptrs(o_seq, n), _ptrs(lse_shards, n), softmax_scale, _stream(stream)),
            "basp_layer_fwd_fused")
+
+
+BASP_STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def basp_layer_fwd_static(plan, q_seq, k_seq, v_seq, o_seq, lse_shards=None, softmax_scale=0.0, stream=None):
+    """The three-launch layer for callers that can neither allocate device memory nor pass a
+    workspace: scratch is a fixed 16 MiB array inside the library (plans that need more are refused).
+    Calls on one device share that array, so do not let two of them overlap on the GPU."""
+    n = plan.N
+    _check(lib.basp_layer_fwd_static(plan.handle, _ptrs(q_seq, n), _ptrs(k_seq, n), _ptrs(v_seq, n),
+                                     _ptrs(o_seq, n), _ptrs(lse_shards, n), softmax_scale, _stream(stream)),
+           "basp_layer_fwd_static")
 
 
 def basp_layer_fwd_host(plan, q_seq_host, k_seq_host, v_seq_host, o_seq_host, device_arena, softmax_scale=0.0,
