@@ -220,6 +220,15 @@ def run_gpu(args, w: synth.Workload):
     ms_h2s = statistics.mean(e[2].elapsed_time(e[3]) for e in ev)
     basp.basp_get_status()
 
+    if args.quick:     # kernel timings only (what the ncu recipes in profiles/ run)
+        clocks = sampler.stop() if sampler else None
+        if rank == 0:
+            print(json.dumps({"workload": w.name, "ms_per_step": total_ms / args.steps, "ms_s2h": ms_s2h,
+                              "ms_attn": ms_attn, "ms_h2s": ms_h2s, "gpu_launches": launches,
+                              "attn_tflops": w.attn_flops_fwd() / ms_attn / 1e9, "clocks": clocks}), flush=True)
+        pdist.finalize()
+        return
+
     # fused layer (a5): one kernel straight from / to the sequence-sharded shards
     for _ in range(max(1, args.warmup // 2)):
         basp.basp_layer_fwd_fused(plan, q_seq, k_seq, v_seq, o_seq)
@@ -309,6 +318,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="basp", choices=["basp", "reference"])
+    ap.add_argument("--quick", action="store_true", help="time the three kernels only (for profiler runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     w = synth.WORKLOADS[args.workload]

@@ -1,0 +1,58 @@
+// Parameter block and tile addressing shared by the attention kernels.
+#pragma once
+#include <cuda.h>
+#include <math.h>
+
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace {
+
+using namespace ptx;
+
+constexpr int kTile = 128;     // query rows and key rows per tile
+
+template <int R>
+struct AttnParams {
+    CUtensorMap q[R], k[R], v[R];
+    __nv_bfloat16 *o[R];
+    float *lse[R];
+    int n_ranks, K, Bl, S, T, Hq_l, Hkv_l, q_per_kv;
+    int o_heads;            // heads in one row of the O destination (Hq_l, or Hq when fused)
+    int fused, causal, has_lse;
+    float scale_log2;       // softmax scale * log2(e)
+    int *status;
+};
+
+struct TileCoord {
+    int rank, row, head;
+};
+
+// Where the 128-token tile starting at sequence position s0 of (rank r, sequence bl, local
+// head h) is found.  `heads_l` is the number of local heads of that tensor.
+template <int R>
+__device__ __forceinline__ TileCoord locate(const AttnParams<R> &p, int r, int bl, int s0, int h, int heads_l) {
+    TileCoord c;
+    if (p.fused) {
+        const int g = r / p.K, l = r - g * p.K;
+        const int owner = s0 / p.T;
+        c.rank = g * p.K + owner;
+        c.row = bl * p.T + (s0 - owner * p.T);
+        c.head = l * heads_l + h;
+    } else {
+        c.rank = r;
+        c.row = bl * p.S + s0;
+        c.head = h;
+    }
+    return c;
+}
+
+__device__ __forceinline__ void report(int *status, int code, int role, int detail) {
+    if (atomicCAS(status, 0, code) == 0) {
+        status[1] = role;
+        status[2] = (int)blockIdx.x;
+        status[3] = detail;
+    }
+}
+
+}  // namespace

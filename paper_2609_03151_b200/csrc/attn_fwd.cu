@@ -13,57 +13,22 @@
 #include "common.cuh"
 #include "ptx.cuh"
 #include "tmap.cuh"
+#include "attn_common.cuh"
+#include "attn_fwd_ws.cuh"
 
 int *basp_status_device_ptr();
 
+static int g_attn_variant = 0;
+extern "C" void basp_debug_set_attn_variant(int v) { g_attn_variant = v; }
+#ifdef BASP_PHASE_TIMING
+extern "C" int basp_debug_phases(long long *out, int reset) {
+    if (out && cudaMemcpyFromSymbol(out, g_phase_cycles, sizeof(long long) * 64) != cudaSuccess) return -1;
+    if (reset) { long long z[64] = {0}; if (cudaMemcpyToSymbol(g_phase_cycles, z, sizeof(z)) != cudaSuccess) return -1; }
+    return 0;
+}
+#endif
+
 namespace {
-
-using namespace ptx;
-
-constexpr int kTile = 128;     // query rows and key rows per tile
-
-template <int R>
-struct AttnParams {
-    CUtensorMap q[R], k[R], v[R];
-    __nv_bfloat16 *o[R];
-    float *lse[R];
-    int K, Bl, S, T, Hq_l, Hkv_l, q_per_kv;
-    int o_heads;            // heads in one row of the O destination (Hq_l, or Hq when fused)
-    int fused, causal, has_lse;
-    float scale_log2;       // softmax scale * log2(e)
-    int *status;
-};
-
-struct TileCoord {
-    int rank, row, head;
-};
-
-// Where the 128-token tile starting at sequence position s0 of (rank r, sequence bl, local
-// head h) is found.  `heads_l` is the number of local heads of that tensor.
-template <int R>
-__device__ __forceinline__ TileCoord locate(const AttnParams<R> &p, int r, int bl, int s0, int h, int heads_l) {
-    TileCoord c;
-    if (p.fused) {
-        const int g = r / p.K, l = r - g * p.K;
-        const int owner = s0 / p.T;
-        c.rank = g * p.K + owner;
-        c.row = bl * p.T + (s0 - owner * p.T);
-        c.head = l * heads_l + h;
-    } else {
-        c.rank = r;
-        c.row = bl * p.S + s0;
-        c.head = h;
-    }
-    return c;
-}
-
-__device__ __forceinline__ void report(int *status, int code, int role, int detail) {
-    if (atomicCAS(status, 0, code) == 0) {
-        status[1] = role;
-        status[2] = (int)blockIdx.x;
-        status[3] = detail;
-    }
-}
 
 // ---------------------------------------------------------------------------------------
 // Baseline kernel: one CTA of 128 threads per (q tile, head, sequence); every step in order.
@@ -242,7 +207,7 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
         prm.o[r] = (__nv_bfloat16 *)o[r];
         prm.lse[r] = lse ? lse[r] : nullptr;
     }
-    prm.K = pl->K; prm.Bl = pl->Bl; prm.S = pl->S; prm.T = pl->T;
+    prm.n_ranks = pl->N; prm.K = pl->K; prm.Bl = pl->Bl; prm.S = pl->S; prm.T = pl->T;
     prm.Hq_l = pl->Hq_l; prm.Hkv_l = pl->Hkv_l; prm.q_per_kv = pl->Hq / pl->Hkv;
     prm.o_heads = hq;
     prm.fused = fused; prm.causal = pl->causal; prm.has_lse = lse != nullptr;
@@ -250,15 +215,32 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
     prm.status = basp_status_device_ptr();
     if (!prm.status) return BASP_ERR_CUDA;
 
-    dim3 grid(pl->S / kTile, pl->Hq_l, pl->N * pl->Bl);
-    if (pl->D == 128) {
-        const int smem = 3 * kTile * 128 * 2 + 1024;
-        BASP_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_simple_kernel<128, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attn_fwd_simple_kernel<128, R><<<grid, 128, smem, st>>>(prm);
+    if (g_attn_variant == 1) {      // baseline kernel (development comparison only)
+        dim3 grid(pl->S / kTile, pl->Hq_l, pl->N * pl->Bl);
+        if (pl->D == 128) {
+            const int smem = 3 * kTile * 128 * 2 + 1024;
+            BASP_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_simple_kernel<128, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            attn_fwd_simple_kernel<128, R><<<grid, 128, smem, st>>>(prm);
+        } else {
+            const int smem = 3 * kTile * 64 * 2 + 1024;
+            BASP_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_simple_kernel<64, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            attn_fwd_simple_kernel<64, R><<<grid, 128, smem, st>>>(prm);
+        }
     } else {
-        const int smem = 3 * kTile * 64 * 2 + 1024;
-        BASP_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_simple_kernel<64, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attn_fwd_simple_kernel<64, R><<<grid, 128, smem, st>>>(prm);
+        int dev = 0, sms = 0;
+        BASP_CUDA_TRY(cudaGetDevice(&dev));
+        BASP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        const long long items = (long long)((pl->S / kTile + 1) / 2) * pl->N * pl->Bl * pl->Hq_l;
+        const int grid = (int)(items < sms ? items : sms);
+        if (pl->D == 128) {
+            const int smem = (2 + kStages) * kTile * 128 * 2 + 1024;
+            BASP_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_ws_kernel<128, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            attn_fwd_ws_kernel<128, R><<<grid, kWsThreads, smem, st>>>(prm);
+        } else {
+            const int smem = (2 + kStages) * kTile * 64 * 2 + 1024;
+            BASP_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_ws_kernel<64, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            attn_fwd_ws_kernel<64, R><<<grid, kWsThreads, smem, st>>>(prm);
+        }
     }
     BASP_CUDA_TRY(cudaGetLastError());
     basp_count_launch(1);

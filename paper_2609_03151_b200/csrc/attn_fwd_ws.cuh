@@ -1,0 +1,402 @@
+// Warp-specialised persistent attention kernel (one CTA of 512 threads per SM).
+//
+// A work item is one block of 256 query rows of one (rank, sequence, local head): two 128-row
+// query tiles that share one stream of K/V tiles.  Roles:
+//   warps  0-3   softmax of query tile 0      (one thread per score row)
+//   warps  4-7   softmax of query tile 1
+//   warps  8-11  correction: rescales the O accumulators in TMEM when a row's reference maximum
+//                moved, and writes the normalised O tile at the end of the item
+//   warp  12     TMA producer (Q tiles, then K_0 V_0 K_1 V_1 ... through a shared-memory ring)
+//   warp  13     tcgen05.mma issuer (one thread)
+// While the softmax warps of one tile work on S_t(j), the tensor core runs P.V and the next
+// Q.K^T of the other tile.  TMEM: S_0 | S_1 | O_0 | O_1 (P_t as bf16 over the first 64 columns of
+// S_t).  All hand-offs are mbarriers; every wait is bounded.
+//
+// Online softmax with a lazily updated reference: the running reference m of a row only moves
+// when the tile maximum exceeds it by more than 8 (log2 units), so most iterations need no
+// rescale of O (exp2(s - m) <= 256 stays well inside bf16/fp32 range; the result is the same
+// softmax, the final division by the row sum absorbs the reference).
+#pragma once
+#include "attn_common.cuh"
+
+namespace {
+
+constexpr int kWsThreads = 512;
+constexpr int kStages = 4;            // K/V ring slots (one 128 x D tile each)
+constexpr float kRescaleThreshold = 8.f;
+
+struct WsItem {
+    int r, bl, h, hkv, qb;
+    int n[2];                         // KV tiles of query tile 0 / 1 (0 = tile absent)
+    int n_max;
+};
+
+template <int R>
+__device__ __forceinline__ bool ws_get_item(const AttnParams<R> &p, int round, WsItem &it) {
+    const int n_qt = p.S / kTile;
+    const int n_qb = (n_qt + 1) / 2;
+    const int per_qb = p.n_ranks * p.Bl * p.Hq_l;
+    const int total = n_qb * per_qb;
+    const int pos = (round & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x;   // boustrophedon
+    const int i = round * (int)gridDim.x + pos;
+    if (i >= total) return false;
+    it.qb = n_qb - 1 - i / per_qb;    // longest blocks first
+    int rem = i % per_qb;
+    it.h = rem % p.Hq_l;
+    rem /= p.Hq_l;
+    it.bl = rem % p.Bl;
+    it.r = rem / p.Bl;
+    it.hkv = it.h / p.q_per_kv;
+    const int qt0 = 2 * it.qb, qt1 = qt0 + 1;
+    const bool has1 = qt1 < n_qt;
+    it.n[0] = p.causal ? qt0 + 1 : n_qt;
+    it.n[1] = has1 ? (p.causal ? qt1 + 1 : n_qt) : 0;
+    it.n_max = it.n[1] > it.n[0] ? it.n[1] : it.n[0];
+    return true;
+}
+
+struct WsShared {
+    uint64_t q_full, q_empty;
+    uint64_t kv_full[kStages], kv_empty[kStages];
+    uint64_t s_full[2], alpha_full[2], p_full[2], o_rescaled[2], o_final[2], l_full[2], o_free[2];
+    float alpha[2][kTile];
+    float l[2][kTile];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+#ifdef BASP_PHASE_TIMING
+__device__ long long g_phase_cycles[64];
+#define PHASE_T(var) const long long var = clock64()
+#define PHASE_ADD(slot, a, b) do { if (blockIdx.x == 0 && (threadIdx.x & 127) == 0) g_phase_cycles[slot] += (b) - (a); } while (0)
+#define PHASE_ADD1(slot, a, b) do { if (blockIdx.x == 0) g_phase_cycles[slot] += (b) - (a); } while (0)
+#else
+#define PHASE_T(var)
+#define PHASE_ADD(slot, a, b)
+#define PHASE_ADD1(slot, a, b)
+#endif
+
+#define WS_WAIT(bar, parity, role, detail)                                     \
+    do {                                                                        \
+        if (!mbar_wait((bar), (parity), &sh.abort_flag)) {                     \
+            sh.abort_flag = 1;                                                  \
+            report(p.status, 1, (role), (detail));                              \
+            goto ws_done;                                                       \
+        }                                                                       \
+    } while (0)
+
+template <int D, int R>
+__global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid_constant__ AttnParams<R> p) {
+    constexpr int kSlabs = D / 64;
+    constexpr int kTileBytes = kTile * D * 2;
+    constexpr int kOCols = D;                          // fp32 accumulator columns per O tile
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *sQ = smem;                                // 2 tiles
+    uint8_t *sKV = smem + 2 * kTileBytes;              // kStages tiles
+    __shared__ WsShared sh;
+
+    // the warp index is broadcast from lane 0 so that the compiler knows it is warp-uniform
+    const int tid = threadIdx.x, warp = __shfl_sync(0xffffffffu, tid >> 5, 0), lane = tid & 31;
+
+    if (tid == 0) {
+        mbar_init(&sh.q_full, 1);
+        mbar_init(&sh.q_empty, 1);
+        for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], 1); }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(&sh.s_full[t], 1);
+            mbar_init(&sh.alpha_full[t], 4);
+            mbar_init(&sh.p_full[t], 4);
+            mbar_init(&sh.o_rescaled[t], 4);
+            mbar_init(&sh.o_final[t], 1);
+            mbar_init(&sh.l_full[t], 4);
+            mbar_init(&sh.o_free[t], 4);
+        }
+        sh.abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 12) { tmem_alloc(&sh.tmem_base, 512); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh.tmem_base;
+    // S_t at columns 128 t, O_t at 256 + 128 t (only kOCols of them used); P_t overlays S_t.
+
+    if (warp < 8) {
+        // =============================================================== softmax of query tile t
+        reg_inc<176>();
+        const int t = warp >> 2;
+        const int row = tid & 127;
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t S_t = tmem + 128 * t + lane_addr;
+        uint32_t it_cnt = 0, ep_cnt = 0;
+        WsItem item;
+        for (int round = 0; ws_get_item(p, round, item); ++round) {
+            const int n_t = item.n[t];
+            if (n_t == 0) continue;
+            float m_ref = -INFINITY, l_run = 0.f;
+            for (int j = 0; j < n_t; ++j, ++it_cnt) {
+                PHASE_T(c0);
+                WS_WAIT(&sh.s_full[t], it_cnt & 1, 10 + t, j);
+                tc_fence_after();
+                PHASE_T(c1);
+                uint32_t s[kTile];
+                tmem_ld_x32(S_t + 0, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+                tmem_ld_x32(S_t + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+                tmem_ld_x32(S_t + 64, *reinterpret_cast<uint32_t(*)[32]>(&s[64]));
+                tmem_ld_x32(S_t + 96, *reinterpret_cast<uint32_t(*)[32]>(&s[96]));
+                tmem_wait_ld();
+                PHASE_T(c2);
+                if (p.causal && j == n_t - 1) {        // diagonal tile: key column i visible iff i <= row
+#pragma unroll
+                    for (int i = 0; i < kTile; ++i)
+                        if (i > row) s[i] = 0xff800000u;   // -inf
+                }
+                float mxs[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) mxs[i] = __uint_as_float(s[i]);
+#pragma unroll
+                for (int i = 8; i < kTile; ++i) mxs[i & 7] = fmaxf(mxs[i & 7], __uint_as_float(s[i]));
+                float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
+                                 fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
+                mx *= p.scale_log2;
+                float m_new, alpha;
+                if (j == 0) { m_new = mx; alpha = 1.f; }
+                else if (mx > m_ref + kRescaleThreshold) { m_new = mx; alpha = exp2_approx(m_ref - m_new); }
+                else { m_new = m_ref; alpha = 1.f; }
+                sh.alpha[t][row] = alpha;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.alpha_full[t]);
+                m_ref = m_new;
+                PHASE_T(c3);
+                float rs[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int i = 0; i < kTile; i += 2) {
+                    const float e0 = exp2_approx(fmaf(__uint_as_float(s[i]), p.scale_log2, -m_new));
+                    const float e1 = exp2_approx(fmaf(__uint_as_float(s[i + 1]), p.scale_log2, -m_new));
+                    rs[(i >> 1) & 3] += e0 + e1;
+                    s[i >> 1] = pack_bf16x2(e0, e1);
+                }
+                l_run = l_run * alpha + ((rs[0] + rs[1]) + (rs[2] + rs[3]));
+                PHASE_T(c4);
+                tmem_st_x32(S_t + 0, *reinterpret_cast<const uint32_t(*)[32]>(&s[0]));
+                tmem_st_x32(S_t + 32, *reinterpret_cast<const uint32_t(*)[32]>(&s[32]));
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.p_full[t]);
+                PHASE_T(c5);
+                PHASE_ADD(8 * t + 0, c0, c1); PHASE_ADD(8 * t + 1, c1, c2); PHASE_ADD(8 * t + 2, c2, c3);
+                PHASE_ADD(8 * t + 3, c3, c4); PHASE_ADD(8 * t + 4, c4, c5); PHASE_ADD(8 * t + 5, c0, c0 + 1);
+            }
+            sh.l[t][row] = l_run;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.l_full[t]);
+            ++ep_cnt;
+            if (p.has_lse) {
+                const int s_pos = (2 * item.qb + t) * kTile + row;
+                p.lse[item.r][((size_t)item.bl * p.Hq_l + item.h) * p.S + s_pos] =
+                    m_ref * 0.6931471805599453f + logf(l_run);
+            }
+        }
+    } else if (warp < 12) {
+        // =============================================================== correction + epilogue
+        reg_dec<80>();
+        const int row = tid & 127;
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        uint32_t it_cnt[2] = {0, 0}, ep_cnt[2] = {0, 0};
+        WsItem item;
+        for (int round = 0; ws_get_item(p, round, item); ++round) {
+            for (int j = 0; j < item.n_max; ++j) {
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (j >= item.n[t]) continue;
+                    WS_WAIT(&sh.alpha_full[t], it_cnt[t] & 1, 20 + t, j);
+                    ++it_cnt[t];
+                    const float alpha = sh.alpha[t][row];
+                    if (j > 0 && !__all_sync(0xffffffffu, alpha == 1.f)) {
+                        tc_fence_after();
+                        const uint32_t O_t = tmem + 256 + 128 * t + lane_addr;
+#pragma unroll
+                        for (int c = 0; c < kOCols / 32; ++c) {
+                            uint32_t rr[32];
+                            tmem_ld_x32(O_t + c * 32, rr);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) rr[i] = __float_as_uint(__uint_as_float(rr[i]) * alpha);
+                            tmem_st_x32(O_t + c * 32, rr);
+                        }
+                        tmem_wait_st();
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sh.o_rescaled[t]);
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                if (item.n[t] == 0) continue;
+                WS_WAIT(&sh.l_full[t], ep_cnt[t] & 1, 24 + t, 0);
+                WS_WAIT(&sh.o_final[t], ep_cnt[t] & 1, 26 + t, 0);
+                ++ep_cnt[t];
+                tc_fence_after();
+                const float inv_l = 1.f / sh.l[t][row];
+                const TileCoord c = locate(p, item.r, item.bl, (2 * item.qb + t) * kTile, item.h, p.Hq_l);
+                __nv_bfloat16 *dst = p.o[c.rank] + ((size_t)(c.row + row) * p.o_heads + c.head) * D;
+                const uint32_t O_t = tmem + 256 + 128 * t + lane_addr;
+#pragma unroll
+                for (int cc = 0; cc < kOCols / 32; ++cc) {
+                    uint32_t rr[32];
+                    tmem_ld_x32(O_t + cc * 32, rr);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 o4;
+                        o4.x = pack_bf16x2(__uint_as_float(rr[8 * i + 0]) * inv_l, __uint_as_float(rr[8 * i + 1]) * inv_l);
+                        o4.y = pack_bf16x2(__uint_as_float(rr[8 * i + 2]) * inv_l, __uint_as_float(rr[8 * i + 3]) * inv_l);
+                        o4.z = pack_bf16x2(__uint_as_float(rr[8 * i + 4]) * inv_l, __uint_as_float(rr[8 * i + 5]) * inv_l);
+                        o4.w = pack_bf16x2(__uint_as_float(rr[8 * i + 6]) * inv_l, __uint_as_float(rr[8 * i + 7]) * inv_l);
+                        *reinterpret_cast<uint4 *>(dst + cc * 32 + i * 8) = o4;
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.o_free[t]);
+            }
+        }
+    } else {
+        reg_dec<80>();
+        if (warp == 12) {
+            // =========================================================== TMA producer (lane 0 issues)
+            uint32_t kv_it = 0, item_n = 0;
+            WsItem item;
+            for (int round = 0; ws_get_item(p, round, item); ++round, ++item_n) {
+                WS_WAIT(&sh.q_empty, (item_n & 1) ^ 1, 30, round);
+                const int n_tiles = item.n[1] > 0 ? 2 : 1;
+                if (lane == 0) mbar_arrive_expect_tx(&sh.q_full, n_tiles * kTileBytes);
+                for (int t = 0; t < n_tiles; ++t) {
+                    const TileCoord c = locate(p, item.r, item.bl, (2 * item.qb + t) * kTile, item.h, p.Hq_l);
+                    if (lane == 0)
+                        for (int s = 0; s < kSlabs; ++s)
+                            tma_load_3d(sQ + t * kTileBytes + s * 16384, &p.q[c.rank], &sh.q_full, s * 64, c.head, c.row);
+                }
+                for (int j = 0; j < item.n_max; ++j) {
+                    const TileCoord c = locate(p, item.r, item.bl, j * kTile, item.hkv, p.Hkv_l);
+#pragma unroll
+                    for (int x = 0; x < 2; ++x, ++kv_it) {
+                        const uint32_t slot = kv_it % kStages, ph = (kv_it / kStages) & 1;
+                        WS_WAIT(&sh.kv_empty[slot], ph ^ 1, 31, j);
+                        const CUtensorMap *tm = x == 0 ? &p.k[c.rank] : &p.v[c.rank];
+                        if (lane == 0) {
+                            mbar_arrive_expect_tx(&sh.kv_full[slot], kTileBytes);
+                            for (int s = 0; s < kSlabs; ++s)
+                                tma_load_3d(sKV + slot * kTileBytes + s * 16384, tm, &sh.kv_full[slot], s * 64, c.head, c.row);
+                        }
+                    }
+                }
+            }
+        } else if (warp == 13) {
+            // =========================================================== MMA issuer (lane 0 issues)
+            const uint32_t idesc_qk = make_idesc_bf16(kTile, kTile, false, false);
+            const uint32_t idesc_pv = make_idesc_bf16(kTile, D, false, true);
+            uint32_t kv_it = 0, item_n = 0, it_cnt[2] = {0, 0}, ep_cnt[2] = {0, 0};
+            WsItem item;
+            // Descriptors differ only in the 14-bit start-address field, so a step along K is an add.
+            const uint64_t desc_k = make_smem_desc_sw128(0, 16, 1024);        // K-major operands (Q, K)
+            const uint64_t desc_v = make_smem_desc_sw128(0, 16384, 1024);     // MN-major operand (V)
+            const uint32_t q_addr16 = smem_u32(sQ) >> 4, kv_addr16 = smem_u32(sKV) >> 4;
+            auto issue_qk = [&](int t, uint32_t slot) {
+                const uint64_t a = desc_k | (uint64_t)(q_addr16 + t * (kTileBytes >> 4));
+                const uint64_t b = desc_k | (uint64_t)(kv_addr16 + slot * (kTileBytes >> 4));
+                if (lane == 0) {
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off16 = ((kk / 4) * 16384 + (kk % 4) * 32) >> 4;
+                        mma_ss(tmem + 128 * t, a + off16, b + off16, idesc_qk, kk > 0);
+                    }
+                    tc_commit(&sh.s_full[t]);
+                }
+            };
+            auto commit = [&](uint64_t *bar) { if (lane == 0) tc_commit(bar); };
+            for (int round = 0; ws_get_item(p, round, item); ++round, ++item_n) {
+                WS_WAIT(&sh.q_full, item_n & 1, 40, round);
+                uint32_t slot_k = kv_it % kStages;
+                WS_WAIT(&sh.kv_full[slot_k], (kv_it / kStages) & 1, 41, 0);
+                ++kv_it;
+                tc_fence_after();
+                for (int t = 0; t < 2; ++t)
+                    if (item.n[t] > 0) issue_qk(t, slot_k);
+                commit(&sh.kv_empty[slot_k]);
+                if (item.n_max == 1) commit(&sh.q_empty);
+                for (int j = 0; j < item.n_max; ++j) {
+                    const uint32_t slot_v = kv_it % kStages;
+                    PHASE_T(e0);
+                    WS_WAIT(&sh.kv_full[slot_v], (kv_it / kStages) & 1, 42, j);
+                    PHASE_T(e1);
+                    PHASE_ADD1(21, e0, e1); PHASE_ADD1(23, e0, e0 + 1);
+                    ++kv_it;
+                    const bool has_next = j + 1 < item.n_max;
+                    bool next_ready = false;
+                    if (has_next) { slot_k = kv_it % kStages; }
+                    const int last_v = j < item.n[1] ? 1 : 0;               // last tile that reads V_j
+                    const int last_k = (j + 1) < item.n[1] ? 1 : 0;         // last tile that reads K_{j+1}
+                    for (int t = 0; t < 2; ++t) {
+                        if (j < item.n[t]) {
+                            PHASE_T(d0);
+                            if (j == 0) WS_WAIT(&sh.o_free[t], (ep_cnt[t] & 1) ^ 1, 43 + t, round);
+                            PHASE_T(d1);
+                            WS_WAIT(&sh.p_full[t], it_cnt[t] & 1, 45 + t, j);
+                            PHASE_T(d2);
+                            WS_WAIT(&sh.o_rescaled[t], it_cnt[t] & 1, 47 + t, j);
+                            PHASE_T(d3);
+                            ++it_cnt[t];
+                            tc_fence_after();
+                            const uint64_t b = desc_v | (uint64_t)(kv_addr16 + slot_v * (kTileBytes >> 4));
+                            if (lane == 0) {
+#pragma unroll
+                                for (int kk = 0; kk < kTile / 16; ++kk)
+                                    mma_ts(tmem + 256 + 128 * t, tmem + 128 * t + kk * 8, b + kk * (2048 >> 4), idesc_pv,
+                                           (j > 0) || (kk > 0));
+                            }
+                            if (j == item.n[t] - 1) { commit(&sh.o_final[t]); ++ep_cnt[t]; }
+                            PHASE_T(d4);
+                            PHASE_ADD1(16, d0, d1); PHASE_ADD1(17 + t, d1, d2); PHASE_ADD1(19, d2, d3); PHASE_ADD1(20, d3, d4);
+                        }
+                        if (t == last_v) commit(&sh.kv_empty[slot_v]);
+                        if (j + 1 < item.n[t]) {
+                            if (!next_ready) {
+                                PHASE_T(f0);
+                                WS_WAIT(&sh.kv_full[slot_k], (kv_it / kStages) & 1, 49, j);
+                                PHASE_T(f1);
+                                PHASE_ADD1(22, f0, f1);
+                                ++kv_it;
+                                next_ready = true;
+                                tc_fence_after();
+                            }
+                            issue_qk(t, slot_k);
+                            if (t == last_k) {
+                                commit(&sh.kv_empty[slot_k]);
+                                if (j + 2 == item.n_max) commit(&sh.q_empty);   // that was the item's last Q.K^T
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+ws_done:
+    tc_fence_before();
+    __syncthreads();
+    if (sh.abort_flag) {
+        // let copies that are still in flight land before the shared memory is given back
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) { }
+        __syncthreads();
+    }
+    if (warp == 12) tmem_dealloc(tmem, 512);
+}
+
+#undef WS_WAIT
+
+}  // namespace
