@@ -19,6 +19,7 @@ struct AttnParams {
     float *lse[R];
     int n_ranks, K, Bl, S, T, Hq_l, Hkv_l, q_per_kv;
     int o_heads;            // heads in one row of the O destination (Hq_l, or Hq when fused)
+    int qb_band;            // query blocks per scheduling band (divides the number of 256-row blocks)
     int fused, causal, has_lse;
     float scale_log2;       // softmax scale * log2(e)
     int *status;

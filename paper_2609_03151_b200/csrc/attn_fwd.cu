@@ -21,6 +21,9 @@ int *basp_status_device_ptr();
 static int g_attn_variant = 0;
 extern "C" void basp_debug_set_attn_variant(int v) { g_attn_variant = v; }
 #ifdef BASP_PHASE_TIMING
+extern "C" int basp_debug_trace(long long *out) {
+    return cudaMemcpyFromSymbol(out, g_trace, sizeof(long long) * 4 * 256) == cudaSuccess ? 0 : -1;
+}
 extern "C" int basp_debug_phases(long long *out, int reset) {
     if (out && cudaMemcpyFromSymbol(out, g_phase_cycles, sizeof(long long) * 64) != cudaSuccess) return -1;
     if (reset) { long long z[64] = {0}; if (cudaMemcpyToSymbol(g_phase_cycles, z, sizeof(z)) != cudaSuccess) return -1; }
@@ -210,6 +213,12 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
     prm.n_ranks = pl->N; prm.K = pl->K; prm.Bl = pl->Bl; prm.S = pl->S; prm.T = pl->T;
     prm.Hq_l = pl->Hq_l; prm.Hkv_l = pl->Hkv_l; prm.q_per_kv = pl->Hq / pl->Hkv;
     prm.o_heads = hq;
+    {
+        const int n_qb = (pl->S / kTile + 1) / 2, q_per_kv = pl->Hq / pl->Hkv;
+        int band = 16 / q_per_kv < 1 ? 1 : (16 / q_per_kv > 8 ? 8 : 16 / q_per_kv);
+        while (n_qb % band != 0) --band;
+        prm.qb_band = band;
+    }
     prm.fused = fused; prm.causal = pl->causal; prm.has_lse = lse != nullptr;
     prm.scale_log2 = (scale == 0.f ? 1.f / sqrtf((float)pl->D) : scale) * 1.4426950408889634f;
     prm.status = basp_status_device_ptr();

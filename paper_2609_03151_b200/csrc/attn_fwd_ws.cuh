@@ -17,6 +17,8 @@
 // rescale of O (exp2(s - m) <= 256 stays well inside bf16/fp32 range; the result is the same
 // softmax, the final division by the row sum absorbs the reference).
 #pragma once
+#include <type_traits>
+
 #include "attn_common.cuh"
 
 namespace {
@@ -24,6 +26,10 @@ namespace {
 constexpr int kWsThreads = 512;
 constexpr int kStages = 4;            // K/V ring slots (one 128 x D tile each)
 constexpr float kRescaleThreshold = 8.f;
+#ifndef BASP_POLY_PAIRS
+#define BASP_POLY_PAIRS 0
+#endif
+constexpr int kPolyPairsOf4 = BASP_POLY_PAIRS;   // of every 4 score pairs, how many take the polynomial exp2
 
 struct WsItem {
     int r, bl, h, hkv, qb;
@@ -40,13 +46,22 @@ __device__ __forceinline__ bool ws_get_item(const AttnParams<R> &p, int round, W
     const int pos = (round & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x;   // boustrophedon
     const int i = round * (int)gridDim.x + pos;
     if (i >= total) return false;
-    it.qb = n_qb - 1 - i / per_qb;    // longest blocks first
-    int rem = i % per_qb;
-    it.h = rem % p.Hq_l;
-    rem /= p.Hq_l;
-    it.bl = rem % p.Bl;
-    it.r = rem / p.Bl;
-    it.hkv = it.h / p.q_per_kv;
+    // Order: bands of `qb_band` consecutive query blocks, longest first; inside a band the items of
+    // one KV stream (rank, sequence, KV head) are adjacent -- qb_band blocks x q_per_kv query heads --
+    // so that the CTAs running side by side read the same K/V tiles through L2.
+    const int per_band = per_qb * p.qb_band;
+    const int band = i / per_band;
+    int rem = i - band * per_band;
+    const int per_stream = p.qb_band * p.q_per_kv;
+    const int stream = rem / per_stream;
+    rem -= stream * per_stream;
+    const int qb_in_band = rem / p.q_per_kv;
+    it.qb = n_qb - 1 - (band * p.qb_band + qb_in_band);
+    it.hkv = stream % p.Hkv_l;
+    it.h = it.hkv * p.q_per_kv + (rem - qb_in_band * p.q_per_kv);
+    const int sb = stream / p.Hkv_l;
+    it.bl = sb % p.Bl;
+    it.r = sb / p.Bl;
     const int qt0 = 2 * it.qb, qt1 = qt0 + 1;
     const bool has1 = qt1 < n_qt;
     it.n[0] = p.causal ? qt0 + 1 : n_qt;
@@ -70,7 +85,14 @@ __device__ long long g_phase_cycles[64];
 #define PHASE_T(var) const long long var = clock64()
 #define PHASE_ADD(slot, a, b) do { if (blockIdx.x == 0 && (threadIdx.x & 127) == 0) g_phase_cycles[slot] += (b) - (a); } while (0)
 #define PHASE_ADD1(slot, a, b) do { if (blockIdx.x == 0) g_phase_cycles[slot] += (b) - (a); } while (0)
+__device__ long long g_trace[4][256];
+// record (event id, clock) of iterations 200..205 of a role's leader thread in CTA 0
+#define TRACE(role, iter, ev) do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (iter) >= 200 && (iter) < 206 && tr_n < 127) { \
+    g_trace[role][2 * tr_n] = (ev) + 100 * (long long)(iter); g_trace[role][2 * tr_n + 1] = clock64(); ++tr_n; } } while (0)
+#define TRACE_DECL int tr_n = 0
 #else
+#define TRACE(role, iter, ev)
+#define TRACE_DECL
 #define PHASE_T(var)
 #define PHASE_ADD(slot, a, b)
 #define PHASE_ADD1(slot, a, b)
@@ -130,6 +152,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t S_t = tmem + 128 * t + lane_addr;
         uint32_t it_cnt = 0, ep_cnt = 0;
+        TRACE_DECL;
         WsItem item;
         for (int round = 0; ws_get_item(p, round, item); ++round) {
             const int n_t = item.n[t];
@@ -140,6 +163,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 WS_WAIT(&sh.s_full[t], it_cnt & 1, 10 + t, j);
                 tc_fence_after();
                 PHASE_T(c1);
+                if ((warp & 3) == 0) TRACE(t, it_cnt, 1);
                 uint32_t s[kTile];
                 tmem_ld_x32(S_t + 0, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
                 tmem_ld_x32(S_t + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
@@ -147,6 +171,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 tmem_ld_x32(S_t + 96, *reinterpret_cast<uint32_t(*)[32]>(&s[96]));
                 tmem_wait_ld();
                 PHASE_T(c2);
+                if ((warp & 3) == 0) TRACE(t, it_cnt, 2);
                 if (p.causal && j == n_t - 1) {        // diagonal tile: key column i visible iff i <= row
 #pragma unroll
                     for (int i = 0; i < kTile; ++i)
@@ -154,12 +179,18 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 }
                 float mxs[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) mxs[i] = __uint_as_float(s[i]);
+                for (int i = 0; i < 8; ++i) mxs[i] = max3(__uint_as_float(s[i]), __uint_as_float(s[8 + i]), __uint_as_float(s[16 + i]));
 #pragma unroll
-                for (int i = 8; i < kTile; ++i) mxs[i & 7] = fmaxf(mxs[i & 7], __uint_as_float(s[i]));
+                for (int i = 24; i + 15 < kTile; i += 16)
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        mxs[k] = max3(mxs[k], __uint_as_float(s[i + k]), __uint_as_float(s[i + 8 + k]));
+#pragma unroll
+                for (int k = 0; k < 8; ++k) mxs[k] = fmaxf(mxs[k], __uint_as_float(s[120 + k]));
                 float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
                                  fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
                 mx *= p.scale_log2;
+                if ((warp & 3) == 0) TRACE(t, it_cnt, 3);
                 float m_new, alpha;
                 if (j == 0) { m_new = mx; alpha = 1.f; }
                 else if (mx > m_ref + kRescaleThreshold) { m_new = mx; alpha = exp2_approx(m_ref - m_new); }
@@ -169,16 +200,38 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 if (lane == 0) mbar_arrive(&sh.alpha_full[t]);
                 m_ref = m_new;
                 PHASE_T(c3);
-                float rs[4] = {0.f, 0.f, 0.f, 0.f};
+                if ((warp & 3) == 0) TRACE(t, it_cnt, 4);
+                const uint64_t sc2 = pack_f2(p.scale_log2, p.scale_log2), nm2 = pack_f2(-m_new, -m_new);
+                uint64_t rs2[2] = {0ull, 0ull};
+                auto exp_row = [&](auto diag_tag) {
+                    constexpr bool kDiag = decltype(diag_tag)::value;
 #pragma unroll
-                for (int i = 0; i < kTile; i += 2) {
-                    const float e0 = exp2_approx(fmaf(__uint_as_float(s[i]), p.scale_log2, -m_new));
-                    const float e1 = exp2_approx(fmaf(__uint_as_float(s[i + 1]), p.scale_log2, -m_new));
-                    rs[(i >> 1) & 3] += e0 + e1;
-                    s[i >> 1] = pack_bf16x2(e0, e1);
-                }
-                l_run = l_run * alpha + ((rs[0] + rs[1]) + (rs[2] + rs[3]));
+                    for (int i = 0; i < kTile; i += 2) {
+                        const uint64_t x2 = fma2(pack_f2(__uint_as_float(s[i]), __uint_as_float(s[i + 1])), sc2, nm2);
+                        float e0, e1;
+                        if (((i >> 1) & 3) < kPolyPairsOf4) {
+                            exp2_poly_pair(x2, e0, e1);
+                        } else {
+                            float x0, x1;
+                            unpack_f2(x2, x0, x1);
+                            e0 = exp2_approx(x0);
+                            e1 = exp2_approx(x1);
+                        }
+                        if (kDiag) {                  // masked keys contribute exactly nothing
+                            if (i > row) e0 = 0.f;
+                            if (i + 1 > row) e1 = 0.f;
+                        }
+                        rs2[(i >> 1) & 1] = add2(rs2[(i >> 1) & 1], pack_f2(e0, e1));
+                        s[i >> 1] = pack_bf16x2(e0, e1);
+                    }
+                };
+                if (p.causal && j == n_t - 1) exp_row(std::true_type{});
+                else exp_row(std::false_type{});
+                float ra, rb;
+                unpack_f2(add2(rs2[0], rs2[1]), ra, rb);
+                l_run = l_run * alpha + (ra + rb);
                 PHASE_T(c4);
+                if ((warp & 3) == 0) TRACE(t, it_cnt, 5);
                 tmem_st_x32(S_t + 0, *reinterpret_cast<const uint32_t(*)[32]>(&s[0]));
                 tmem_st_x32(S_t + 32, *reinterpret_cast<const uint32_t(*)[32]>(&s[32]));
                 tmem_wait_st();
@@ -186,6 +239,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.p_full[t]);
                 PHASE_T(c5);
+                if ((warp & 3) == 0) TRACE(t, it_cnt, 6);
                 PHASE_ADD(8 * t + 0, c0, c1); PHASE_ADD(8 * t + 1, c1, c2); PHASE_ADD(8 * t + 2, c2, c3);
                 PHASE_ADD(8 * t + 3, c3, c4); PHASE_ADD(8 * t + 4, c4, c5); PHASE_ADD(8 * t + 5, c0, c0 + 1);
             }
@@ -300,6 +354,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
             const uint32_t idesc_qk = make_idesc_bf16(kTile, kTile, false, false);
             const uint32_t idesc_pv = make_idesc_bf16(kTile, D, false, true);
             uint32_t kv_it = 0, item_n = 0, it_cnt[2] = {0, 0}, ep_cnt[2] = {0, 0};
+            TRACE_DECL;
             WsItem item;
             // Descriptors differ only in the 14-bit start-address field, so a step along K is an add.
             const uint64_t desc_k = make_smem_desc_sw128(0, 16, 1024);        // K-major operands (Q, K)
@@ -345,10 +400,12 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                             PHASE_T(d0);
                             if (j == 0) WS_WAIT(&sh.o_free[t], (ep_cnt[t] & 1) ^ 1, 43 + t, round);
                             PHASE_T(d1);
+                            TRACE(2, it_cnt[t], 10 + t);
                             WS_WAIT(&sh.p_full[t], it_cnt[t] & 1, 45 + t, j);
                             PHASE_T(d2);
                             WS_WAIT(&sh.o_rescaled[t], it_cnt[t] & 1, 47 + t, j);
                             PHASE_T(d3);
+                            TRACE(2, it_cnt[t], 20 + t);
                             ++it_cnt[t];
                             tc_fence_after();
                             const uint64_t b = desc_v | (uint64_t)(kv_addr16 + slot_v * (kTileBytes >> 4));
@@ -360,6 +417,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                             }
                             if (j == item.n[t] - 1) { commit(&sh.o_final[t]); ++ep_cnt[t]; }
                             PHASE_T(d4);
+                            TRACE(2, it_cnt[t] - 1, 30 + t);
                             PHASE_ADD1(16, d0, d1); PHASE_ADD1(17 + t, d1, d2); PHASE_ADD1(19, d2, d3); PHASE_ADD1(20, d3, d4);
                         }
                         if (t == last_v) commit(&sh.kv_empty[slot_v]);
@@ -374,6 +432,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                                 tc_fence_after();
                             }
                             issue_qk(t, slot_k);
+                            TRACE(2, it_cnt[t] - 1, 40 + t);
                             if (t == last_k) {
                                 commit(&sh.kv_empty[slot_k]);
                                 if (j + 2 == item.n_max) commit(&sh.q_empty);   // that was the item's last Q.K^T
