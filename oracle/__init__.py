@@ -175,6 +175,68 @@ def attn_fwd_rows(Q: np.ndarray, K: np.ndarray, V: np.ndarray, rows: np.ndarray,
     return O, lse
 
 
+def _scale(scale, D):
+    return 1.0 / np.sqrt(D) if scale is None else scale
+
+
+def attn_bwd(Q, K, V, dO, scale: float | None = None, causal: bool = True):
+    """Gradients of attention by the chain rule (see basp_oracle.c).  Q, dO [Bn,S,Hq,D]; K, V
+    [Bn,S,Hkv,D] uint16.  Returns dict(dQ, dK, dV, LSE, DELTA) in fp64 (LSE/DELTA [Bn,Hq,S])."""
+    Q, K, V, dO = (np.ascontiguousarray(a, dtype=np.uint16) for a in (Q, K, V, dO))
+    Bn, S, Hq, D = Q.shape
+    Hkv = K.shape[2]
+    assert dO.shape == Q.shape and K.shape == (Bn, S, Hkv, D) and V.shape == K.shape
+    dQ = np.empty(Q.shape, dtype=np.float64)
+    dK = np.empty(K.shape, dtype=np.float64)
+    dV = np.empty(K.shape, dtype=np.float64)
+    LSE = np.empty((Bn, Hq, S), dtype=np.float64)
+    DELTA = np.empty((Bn, Hq, S), dtype=np.float64)
+    _load().oracle_attn_bwd(_p(Q), _p(K), _p(V), _p(dO), _p(dQ), _p(dK), _p(dV), _p(LSE), _p(DELTA), Bn, S, Hq,
+                            Hkv, D, ctypes.c_double(_scale(scale, D)), int(causal))
+    return dict(dQ=dQ, dK=dK, dV=dV, LSE=LSE, DELTA=DELTA)
+
+
+def attn_bwd_dq_rows(Q, K, V, dO, rows, scale: float | None = None, causal: bool = True):
+    """dQ of selected rows; ``rows`` int32 [n,3] of (b, h, i) -> [n, D] fp64."""
+    Q, K, V, dO = (np.ascontiguousarray(a, dtype=np.uint16) for a in (Q, K, V, dO))
+    rows = np.ascontiguousarray(rows, dtype=np.int32).reshape(-1, 3)
+    Bn, S, Hq, D = Q.shape
+    out = np.empty((rows.shape[0], D), dtype=np.float64)
+    _load().oracle_attn_bwd_dq_rows(_p(Q), _p(K), _p(V), _p(dO), _p(rows), rows.shape[0], _p(out), S, Hq,
+                                    K.shape[2], D, ctypes.c_double(_scale(scale, D)), int(causal))
+    return out
+
+
+def attn_bwd_dkdv_tail(Q, K, V, dO, b: int, kv: int, ncols: int, scale: float | None = None):
+    """dK, dV of the last ``ncols`` key positions of (sequence b, KV head kv), causal -> two [ncols, D]."""
+    Q, K, V, dO = (np.ascontiguousarray(a, dtype=np.uint16) for a in (Q, K, V, dO))
+    Bn, S, Hq, D = Q.shape
+    dK = np.empty((ncols, D), dtype=np.float64)
+    dV = np.empty((ncols, D), dtype=np.float64)
+    _load().oracle_attn_bwd_dkdv_tail(_p(Q), _p(K), _p(V), _p(dO), int(b), int(kv), int(ncols), _p(dK), _p(dV),
+                                      S, Hq, K.shape[2], D, ctypes.c_double(_scale(scale, D)))
+    return dK, dV
+
+
+def layer_bwd(Xq, Xk, Xv, XdO, pl: Plan, scale: float | None = None, causal: bool = True):
+    """Backward of the sequence-parallel layer, step by step: partition the four global tensors,
+    all-to-all each to head-sharded, per-rank attention backward, reverse all-to-all of dQ, dK, dV,
+    collect.  Returns dict with head- and sequence-sharded gradients and the global ones."""
+    parts = [s2h(partition(X, pl), pl) for X in (Xq, Xk, Xv, XdO)]
+    qh, kh, vh, doh = parts
+    dqh = np.empty(qh.shape, dtype=np.float64)
+    dkh = np.empty(kh.shape, dtype=np.float64)
+    dvh = np.empty(kh.shape, dtype=np.float64)
+    for r in range(pl.N):
+        g = attn_bwd(qh[r], kh[r], vh[r], doh[r], scale, causal)
+        dqh[r], dkh[r], dvh[r] = g["dQ"], g["dK"], g["dV"]
+    out = dict(dq_head=dqh, dk_head=dkh, dv_head=dvh, do_head=doh)
+    for n, a in (("dq", dqh), ("dk", dkh), ("dv", dvh)):
+        out[n + "_seq"] = h2s(a, pl)
+        out[n + "_global"] = gather(out[n + "_seq"], pl)
+    return out
+
+
 # ------------------------------------------------------------------------- layer
 def layer_fwd(Xq: np.ndarray, Xk: np.ndarray, Xv: np.ndarray, pl: Plan,
               scale: float | None = None, causal: bool = True):

@@ -236,3 +236,177 @@ void oracle_attn_fwd_rows(const uint16_t *Q, const uint16_t *Kt, const uint16_t 
         free(scores);
     }
 }
+
+/* ------------------------------------------------------------------------- */
+/* Backward of the attention equation (Section II-A) by the chain rule, written out:
+ *   P_ij  = exp(scale * q_i.k_j - LSE_i)                    (j visible to i)
+ *   D_i   = dO_i . O_i                                       ("delta")
+ *   dV_j  = sum_i P_ij dO_i
+ *   dP_ij = dO_i . v_j
+ *   dS_ij = P_ij (dP_ij - D_i)
+ *   dQ_i  = scale * sum_j dS_ij k_j
+ *   dK_j  = scale * sum_i dS_ij q_i
+ * dK and dV of a KV head are summed over the Hq/Hkv query heads that read it.
+ * Two literal passes: rows (LSE, O, D, dQ), then columns (dK, dV), each recomputing P from
+ * the first pass's LSE.  dO is bf16 bits like the inputs.  Outputs fp64:
+ *   dQ [Bn][S][Hq][D], dK, dV [Bn][S][Hkv][D]. */
+static void bwd_row_stats(const uint16_t *Q, const uint16_t *Kt, const uint16_t *V, const uint16_t *dO,
+                          int S, int Hq, int Hkv, int D, double scale, int causal, int b, int h, int i,
+                          double *scores, double *o_row, double *lse, double *delta) {
+    attn_row(Q, Kt, V, S, Hq, Hkv, D, scale, causal, b, h, i, scores, o_row, lse);
+    const uint16_t *go = dO + (((size_t)b * S + i) * Hq + h) * D;
+    double acc = 0.0;
+    for (int d = 0; d < D; ++d) acc += bf16_to_f64(go[d]) * o_row[d];
+    *delta = acc;
+}
+
+/* dQ of one row, given that row's LSE and delta. */
+static void bwd_dq_row(const uint16_t *Q, const uint16_t *Kt, const uint16_t *V, const uint16_t *dO, int S,
+                       int Hq, int Hkv, int D, double scale, int causal, int b, int h, int i, double lse,
+                       double delta, double *dq_row) {
+    const int kv = h / (Hq / Hkv);
+    const int n = causal ? i + 1 : S;
+    const uint16_t *q = Q + (((size_t)b * S + i) * Hq + h) * D;
+    const uint16_t *go = dO + (((size_t)b * S + i) * Hq + h) * D;
+    for (int d = 0; d < D; ++d) dq_row[d] = 0.0;
+    for (int j = 0; j < n; ++j) {
+        const uint16_t *k = Kt + (((size_t)b * S + j) * Hkv + kv) * D;
+        const uint16_t *v = V + (((size_t)b * S + j) * Hkv + kv) * D;
+        double s = 0.0, dp = 0.0;
+        for (int d = 0; d < D; ++d) {
+            s += bf16_to_f64(q[d]) * bf16_to_f64(k[d]);
+            dp += bf16_to_f64(go[d]) * bf16_to_f64(v[d]);
+        }
+        const double p = exp(s * scale - lse);
+        const double ds = p * (dp - delta);
+        for (int d = 0; d < D; ++d) dq_row[d] += scale * ds * bf16_to_f64(k[d]);
+    }
+}
+
+/* dK and dV of one key column j of KV head kv: sums over the query heads of the group and the
+ * rows that see j.  LSE, DELTA are [Bn][Hq][S]. */
+static void bwd_dkdv_col(const uint16_t *Q, const uint16_t *Kt, const uint16_t *V, const uint16_t *dO,
+                         const double *LSE, const double *DELTA, int S, int Hq, int Hkv, int D, double scale,
+                         int causal, int b, int kv, int j, double *dk_row, double *dv_row) {
+    const int rep = Hq / Hkv;
+    const uint16_t *k = Kt + (((size_t)b * S + j) * Hkv + kv) * D;
+    const uint16_t *v = V + (((size_t)b * S + j) * Hkv + kv) * D;
+    for (int d = 0; d < D; ++d) dk_row[d] = dv_row[d] = 0.0;
+    for (int h = kv * rep; h < (kv + 1) * rep; ++h)
+        for (int i = causal ? j : 0; i < S; ++i) {
+            const uint16_t *q = Q + (((size_t)b * S + i) * Hq + h) * D;
+            const uint16_t *go = dO + (((size_t)b * S + i) * Hq + h) * D;
+            double s = 0.0, dp = 0.0;
+            for (int d = 0; d < D; ++d) {
+                s += bf16_to_f64(q[d]) * bf16_to_f64(k[d]);
+                dp += bf16_to_f64(go[d]) * bf16_to_f64(v[d]);
+            }
+            const double p = exp(s * scale - LSE[((size_t)b * Hq + h) * S + i]);
+            const double ds = p * (dp - DELTA[((size_t)b * Hq + h) * S + i]);
+            for (int d = 0; d < D; ++d) {
+                dv_row[d] += p * bf16_to_f64(go[d]);
+                dk_row[d] += scale * ds * bf16_to_f64(q[d]);
+            }
+        }
+}
+
+void oracle_attn_bwd(const uint16_t *Q, const uint16_t *Kt, const uint16_t *V, const uint16_t *dO, double *dQ,
+                     double *dK, double *dV, double *LSE, double *DELTA, int Bn, int S, int Hq, int Hkv, int D,
+                     double scale, int causal) {
+    const long rows = (long)Bn * Hq * S;
+#pragma omp parallel
+    {
+        double *scores = (double *)malloc(sizeof(double) * (size_t)S);
+        double *o_row = (double *)malloc(sizeof(double) * (size_t)D);
+#pragma omp for schedule(dynamic, 8)
+        for (long r = 0; r < rows; ++r) {
+            const long rr = rows - 1 - r;
+            const int i = (int)(rr % S), h = (int)((rr / S) % Hq), b = (int)(rr / ((long)S * Hq));
+            double lse, delta;
+            bwd_row_stats(Q, Kt, V, dO, S, Hq, Hkv, D, scale, causal, b, h, i, scores, o_row, &lse, &delta);
+            LSE[((size_t)b * Hq + h) * S + i] = lse;
+            DELTA[((size_t)b * Hq + h) * S + i] = delta;
+            bwd_dq_row(Q, Kt, V, dO, S, Hq, Hkv, D, scale, causal, b, h, i, lse, delta,
+                       dQ + (((size_t)b * S + i) * Hq + h) * D);
+        }
+        free(scores);
+        free(o_row);
+    }
+    const long cols = (long)Bn * Hkv * S;
+#pragma omp parallel for schedule(dynamic, 8)
+    for (long c = 0; c < cols; ++c) {
+        const int j = (int)(c % S), kv = (int)((c / S) % Hkv), b = (int)(c / ((long)S * Hkv));
+        bwd_dkdv_col(Q, Kt, V, dO, LSE, DELTA, S, Hq, Hkv, D, scale, causal, b, kv, j,
+                     dK + (((size_t)b * S + j) * Hkv + kv) * D, dV + (((size_t)b * S + j) * Hkv + kv) * D);
+    }
+}
+
+/* Selected dQ rows: rows[3r] = {b, h, i}; dQ_rows [nrows][D]. */
+void oracle_attn_bwd_dq_rows(const uint16_t *Q, const uint16_t *Kt, const uint16_t *V, const uint16_t *dO,
+                             const int *rows, int nrows, double *dQ_rows, int S, int Hq, int Hkv, int D,
+                             double scale, int causal) {
+#pragma omp parallel
+    {
+        double *scores = (double *)malloc(sizeof(double) * (size_t)S);
+        double *o_row = (double *)malloc(sizeof(double) * (size_t)D);
+#pragma omp for schedule(dynamic, 1)
+        for (int r = 0; r < nrows; ++r) {
+            double lse, delta;
+            const int b = rows[3 * r], h = rows[3 * r + 1], i = rows[3 * r + 2];
+            bwd_row_stats(Q, Kt, V, dO, S, Hq, Hkv, D, scale, causal, b, h, i, scores, o_row, &lse, &delta);
+            bwd_dq_row(Q, Kt, V, dO, S, Hq, Hkv, D, scale, causal, b, h, i, lse, delta, dQ_rows + (size_t)r * D);
+        }
+        free(scores);
+        free(o_row);
+    }
+}
+
+/* dK and dV of the LAST ncols key columns (j = S-ncols .. S-1) of (b, kv): only the rows i >= S-ncols
+ * of the group's query heads see them, so the row statistics cost O(ncols * S * D) per head.
+ * dK_cols, dV_cols [ncols][D].  Causal only. */
+void oracle_attn_bwd_dkdv_tail(const uint16_t *Q, const uint16_t *Kt, const uint16_t *V, const uint16_t *dO,
+                               int b, int kv, int ncols, double *dK_cols, double *dV_cols, int S, int Hq,
+                               int Hkv, int D, double scale) {
+    const int rep = Hq / Hkv, i0 = S - ncols;
+    double *lse = (double *)malloc(sizeof(double) * (size_t)rep * ncols);
+    double *delta = (double *)malloc(sizeof(double) * (size_t)rep * ncols);
+#pragma omp parallel
+    {
+        double *scores = (double *)malloc(sizeof(double) * (size_t)S);
+        double *o_row = (double *)malloc(sizeof(double) * (size_t)D);
+#pragma omp for schedule(dynamic, 1)
+        for (int r = 0; r < rep * ncols; ++r) {
+            const int h = kv * rep + r / ncols, i = i0 + r % ncols;
+            bwd_row_stats(Q, Kt, V, dO, S, Hq, Hkv, D, scale, 1, b, h, i, scores, o_row, &lse[r], &delta[r]);
+        }
+        free(scores);
+        free(o_row);
+    }
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int c = 0; c < ncols; ++c) {
+        const int j = i0 + c;
+        const uint16_t *k = Kt + (((size_t)b * S + j) * Hkv + kv) * D;
+        const uint16_t *v = V + (((size_t)b * S + j) * Hkv + kv) * D;
+        double *dk_row = dK_cols + (size_t)c * D, *dv_row = dV_cols + (size_t)c * D;
+        for (int d = 0; d < D; ++d) dk_row[d] = dv_row[d] = 0.0;
+        for (int hh = 0; hh < rep; ++hh)
+            for (int i = j; i < S; ++i) {
+                const int h = kv * rep + hh;
+                const uint16_t *q = Q + (((size_t)b * S + i) * Hq + h) * D;
+                const uint16_t *go = dO + (((size_t)b * S + i) * Hq + h) * D;
+                double s = 0.0, dp = 0.0;
+                for (int d = 0; d < D; ++d) {
+                    s += bf16_to_f64(q[d]) * bf16_to_f64(k[d]);
+                    dp += bf16_to_f64(go[d]) * bf16_to_f64(v[d]);
+                }
+                const double p = exp(s * scale - lse[hh * ncols + (i - i0)]);
+                const double ds = p * (dp - delta[hh * ncols + (i - i0)]);
+                for (int d = 0; d < D; ++d) {
+                    dv_row[d] += p * bf16_to_f64(go[d]);
+                    dk_row[d] += scale * ds * bf16_to_f64(q[d]);
+                }
+            }
+    }
+    free(lse);
+    free(delta);
+}
