@@ -172,6 +172,45 @@ int basp_layer_fwd_fused(const basp_plan *plan, const void *const *q_seq, const 
                          const void *const *v_seq, void *const *o_seq, float *const *lse_shards,
                          float softmax_scale, void *stream);
 
+/* After basp_layer_fwd (or basp_layer_fwd_static) returns, the workspace holds the head-sharded
+ * Q, K, V and O of every rank; this call writes their addresses (n_ranks pointers each) so that a
+ * training step can keep them for the backward pass instead of resharding again. */
+int basp_layer_workspace_shards(const basp_plan *plan, void *workspace, void **q_head, void **k_head,
+                                void **v_head, void **o_head);
+
+/* ---- attention backward over each rank's head slice (the paper trains through this layer but
+ * never writes the backward out; it is the chain rule applied to the Section II-A equation):
+ *   P_ij = exp(scale q_i.k_j - LSE_i),  Delta_i = dO_i.O_i,  dV_j = sum_i P_ij dO_i,
+ *   dS_ij = P_ij (dO_i.v_j - Delta_i),  dQ_i = scale sum_j dS_ij k_j,  dK_j = scale sum_i dS_ij q_i,
+ * with dK, dV summed over the Hq/Hkv query heads of a KV head.  All operands HEAD-sharded: q, o, do, dq
+ * [Bl][S][Hq/K][D]; k, v, dk, dv [Bl][S][Hkv/K][D]; lse as written by the forward.  bf16 in and out,
+ * fp32 accumulation; dQ is accumulated with floating-point atomics, so its last bits may differ
+ * between runs.  Requires D = 128 and S a multiple of 128.  `workspace`: device memory of at least
+ * basp_attn_bwd_workspace_bytes(plan) bytes (fp32 dQ accumulator and Delta). */
+int basp_attn_bwd(const basp_plan *plan, const void *const *q_head, const void *const *k_head,
+                  const void *const *v_head, const void *const *o_head, const void *const *do_head,
+                  const float *const *lse_shards, void *const *dq_head, void *const *dk_head,
+                  void *const *dv_head, void *workspace, size_t workspace_bytes, float softmax_scale,
+                  void *stream);
+size_t basp_attn_bwd_workspace_bytes(const basp_plan *plan);
+
+/* dQ (Hq heads), dK and dV (Hkv heads) head- to sequence-sharded in ONE launch: the reverse
+ * all-to-alls of the gradients. */
+int basp_reshard_grads_h2s(const basp_plan *plan, const void *const *dq_head, const void *const *dk_head,
+                           const void *const *dv_head, void *const *dq_seq, void *const *dk_seq,
+                           void *const *dv_seq, void *stream);
+
+/* ---- backward of the whole layer: all-to-all of dO (sequence- to head-sharded), attention
+ * backward on the saved head-sharded Q, K, V, O and LSE of the forward, reverse all-to-alls of
+ * dQ, dK, dV.  do_seq / dq_seq / dk_seq / dv_seq are SEQUENCE-sharded.  `workspace` of at least
+ * basp_layer_bwd_workspace_bytes(plan) bytes holds the head-sharded dO, dQ, dK, dV and the
+ * attention-backward workspace. */
+int basp_layer_bwd(const basp_plan *plan, const void *const *q_head, const void *const *k_head,
+                   const void *const *v_head, const void *const *o_head, const float *const *lse_shards,
+                   const void *const *do_seq, void *const *dq_seq, void *const *dk_seq, void *const *dv_seq,
+                   void *workspace, size_t workspace_bytes, float softmax_scale, void *stream);
+size_t basp_layer_bwd_workspace_bytes(const basp_plan *plan);
+
 /* ---- the fused layer for callers whose shards are in HOST memory: copies every Q/K/V
  * shard host->device into `device_arena` (device memory, >= basp_host_arena_bytes(plan)
  * bytes), runs basp_layer_fwd_fused, copies every O shard device->host and waits for the

@@ -26,7 +26,9 @@ EXPORTS = [
     "basp_plan_create", "basp_plan_destroy", "basp_plan_get_info", "basp_plan_get_rank",
     "basp_plan_group_ranks", "basp_reshard_s2h", "basp_reshard_h2s", "basp_reshard_qkv_s2h",
     "basp_attn_fwd", "basp_layer_fwd", "basp_workspace_bytes", "basp_layer_fwd_fused",
-    "basp_layer_fwd_host", "basp_host_arena_bytes", "basp_layer_fwd_static", "basp_get_status", "basp_clear_status",
+    "basp_layer_fwd_host", "basp_host_arena_bytes", "basp_layer_fwd_static",
+    "basp_layer_workspace_shards", "basp_attn_bwd", "basp_attn_bwd_workspace_bytes", "basp_reshard_grads_h2s",
+    "basp_layer_bwd", "basp_layer_bwd_workspace_bytes", "basp_get_status", "basp_clear_status",
     "basp_strerror", "basp_last_cuda_error", "basp_launch_count",
 ]
 
@@ -61,6 +63,13 @@ lib.basp_layer_fwd.argtypes = [c_void_p] + [_PP] * 5 + [c_void_p, c_size_t, c_fl
 lib.basp_layer_fwd_fused.argtypes = [c_void_p] + [_PP] * 5 + [c_float, c_void_p]
 lib.basp_layer_fwd_static.argtypes = [c_void_p] + [_PP] * 5 + [c_float, c_void_p]
 lib.basp_layer_fwd_host.argtypes = [c_void_p] + [_PP] * 4 + [c_void_p, c_size_t, c_float, c_void_p]
+lib.basp_layer_workspace_shards.argtypes = [c_void_p, c_void_p] + [_PP] * 4
+lib.basp_attn_bwd.argtypes = [c_void_p] + [_PP] * 9 + [c_void_p, c_size_t, c_float, c_void_p]
+lib.basp_reshard_grads_h2s.argtypes = [c_void_p] + [_PP] * 6 + [c_void_p]
+lib.basp_layer_bwd.argtypes = [c_void_p] + [_PP] * 9 + [c_void_p, c_size_t, c_float, c_void_p]
+for _n in ("basp_attn_bwd_workspace_bytes", "basp_layer_bwd_workspace_bytes"):
+    getattr(lib, _n).argtypes = [c_void_p]
+    getattr(lib, _n).restype = c_size_t
 lib.basp_workspace_bytes.argtypes = [c_void_p]
 lib.basp_workspace_bytes.restype = c_size_t
 lib.basp_host_arena_bytes.argtypes = [c_void_p]
@@ -207,6 +216,63 @@ def basp_layer_fwd_host(plan, q_seq_host, k_seq_host, v_seq_host, o_seq_host, de
                                    _ptrs(o_seq_host, n), c_void_p(device_arena.data_ptr()),
                                    device_arena.numel() * device_arena.element_size(), softmax_scale,
                                    _stream(stream)), "basp_layer_fwd_host")
+
+
+def basp_layer_workspace_shards(plan, workspace):
+    """Addresses (ints) of the head-sharded Q, K, V, O that basp_layer_fwd left in `workspace`:
+    four lists of n_ranks device addresses."""
+    n = plan.N
+    arrs = [(c_void_p * n)() for _ in range(4)]
+    _check(lib.basp_layer_workspace_shards(plan.handle, c_void_p(workspace.data_ptr()), *arrs),
+           "basp_layer_workspace_shards")
+    return [[int(a[i]) for i in range(n)] for a in arrs]
+
+
+class _Addr:
+    """A raw device address standing in for a tensor in the marshalling helpers."""
+
+    def __init__(self, addr):
+        self.addr = addr
+
+    def data_ptr(self):
+        return self.addr
+
+
+def as_shards(addresses):
+    return [_Addr(a) for a in addresses]
+
+
+def basp_attn_bwd_workspace_bytes(plan) -> int:
+    return int(lib.basp_attn_bwd_workspace_bytes(plan.handle))
+
+
+def basp_layer_bwd_workspace_bytes(plan) -> int:
+    return int(lib.basp_layer_bwd_workspace_bytes(plan.handle))
+
+
+def basp_attn_bwd(plan, q_head, k_head, v_head, o_head, do_head, lse_shards, dq_head, dk_head, dv_head, workspace,
+                  softmax_scale=0.0, stream=None):
+    n = plan.N
+    _check(lib.basp_attn_bwd(plan.handle, *[_ptrs(t, n) for t in (q_head, k_head, v_head, o_head, do_head, lse_shards,
+                                                                  dq_head, dk_head, dv_head)],
+                             c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size(),
+                             softmax_scale, _stream(stream)), "basp_attn_bwd")
+
+
+def basp_reshard_grads_h2s(plan, dq_head, dk_head, dv_head, dq_seq, dk_seq, dv_seq, stream=None):
+    n = plan.N
+    _check(lib.basp_reshard_grads_h2s(plan.handle, *[_ptrs(t, n) for t in (dq_head, dk_head, dv_head, dq_seq, dk_seq,
+                                                                           dv_seq)], _stream(stream)),
+           "basp_reshard_grads_h2s")
+
+
+def basp_layer_bwd(plan, q_head, k_head, v_head, o_head, lse_shards, do_seq, dq_seq, dk_seq, dv_seq, workspace,
+                   softmax_scale=0.0, stream=None):
+    n = plan.N
+    _check(lib.basp_layer_bwd(plan.handle, *[_ptrs(t, n) for t in (q_head, k_head, v_head, o_head, lse_shards, do_seq,
+                                                                   dq_seq, dk_seq, dv_seq)],
+                              c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size(),
+                              softmax_scale, _stream(stream)), "basp_layer_bwd")
 
 
 def basp_get_status(stream=None, raise_on_timeout=True):

@@ -173,3 +173,13 @@ extern "C" int basp_reshard_qkv_s2h(const basp_plan *plan, const void *const *q_
                       {plan->Hkv, v_seq, (const void *const *)v_head}};
     return launch(plan, a, 3, true, stream);
 }
+
+extern "C" int basp_reshard_grads_h2s(const basp_plan *plan, const void *const *dq_head, const void *const *dk_head,
+                                      const void *const *dv_head, void *const *dq_seq, void *const *dk_seq,
+                                      void *const *dv_seq, void *stream) {
+    if (!plan) return BASP_ERR_NULL;
+    TensorArg a[3] = {{plan->Hq, (const void *const *)dq_seq, dq_head},
+                      {plan->Hkv, (const void *const *)dk_seq, dk_head},
+                      {plan->Hkv, (const void *const *)dv_seq, dv_head}};
+    return launch(plan, a, 3, false, stream);
+}

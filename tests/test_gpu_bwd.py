@@ -1,0 +1,108 @@
+"""Parity of the attention backward (and the layer backward with its gradient reshards) with the
+fp64 oracle, through the C ABI.
+
+Tolerance for gradients (bf16 operands and outputs, bf16 P and dS, fp32 accumulation): element-wise
+|err| <= 2e-2 + 2^-8 |ref| and mean-abs error <= 2e-3 * max(1, mean |ref|).  dK/dV sum up to S * Hq/Hkv
+terms and exceed magnitude 4, where one bf16 ulp is already 0.016, hence the relative term."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import make_plan, to_dev, to_f64
+from paper_2609_03151_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def assert_grad_close(got, ref, what):
+    err = np.abs(got - ref)
+    bound = 2e-2 + 2.0 ** -8 * np.abs(ref)
+    worst = float((err - bound).max())
+    mean_ok = err.mean() <= 2e-3 * max(1.0, float(np.abs(ref).mean()))
+    assert worst <= 0 and mean_ok, f"{what}: max-abs {err.max():.3e} (excess {worst:.3e}) mean-abs {err.mean():.3e} ref mean {np.abs(ref).mean():.3e}"
+
+
+def inputs(w, seed=0):
+    q, k, v, do = synth.make_qkv(w, seed, with_dO=True)
+    return [synth.bits(t) for t in (q, k, v, do)], oracle.plan(w.N, w.B, w.S, w.G)
+
+
+def run_attn_bwd(basp, w, causal=True, seed=0):
+    (Xq, Xk, Xv, Xdo), op = inputs(w, seed)
+    pl = make_plan(basp, w, causal)
+    qh, kh, vh, doh = (oracle.s2h(oracle.partition(X, op), op) for X in (Xq, Xk, Xv, Xdo))
+    dq_, dk_, dv_, ddo = to_dev(qh), to_dev(kh), to_dev(vh), to_dev(doh)
+    o = [torch.zeros_like(t) for t in dq_]
+    lse = [torch.zeros((op.Bl, w.Hq // op.K, w.S), dtype=torch.float32, device="cuda") for _ in range(w.N)]
+    basp.basp_clear_status()
+    basp.basp_attn_fwd(pl, dq_, dk_, dv_, o, lse)
+    gq = [torch.full_like(t, float("nan")) for t in dq_]
+    gk = [torch.full_like(t, float("nan")) for t in dk_]
+    gv = [torch.full_like(t, float("nan")) for t in dk_]
+    ws = torch.empty(basp.basp_attn_bwd_workspace_bytes(pl), dtype=torch.uint8, device="cuda")
+    basp.basp_attn_bwd(pl, dq_, dk_, dv_, o, ddo, lse, gq, gk, gv, ws)
+    basp.basp_get_status()
+    ref = [oracle.attn_bwd(qh[r], kh[r], vh[r], doh[r], causal=causal) for r in range(w.N)]
+    return (to_f64(gq), to_f64(gk), to_f64(gv)), tuple(np.stack([g[n] for g in ref]) for n in ("dQ", "dK", "dV"))
+
+
+@pytest.mark.parametrize("name,w", [
+    ("one_tile", synth.Workload("one_tile", N=1, B=1, S=128, Hq=1, Hkv=1, D=128)),
+    ("gqa4", synth.Workload("gqa4", N=1, B=1, S=384, Hq=4, Hkv=1, D=128)),
+    ("llama_T128", synth.shrink(synth.WORKLOADS["llama3_8b_128k_train"], 128)),
+    ("llama_b2_T256", synth.shrink(synth.WORKLOADS["llama3_8b_32k"], 256)),
+    ("ulysses", synth.Workload("ulysses", N=4, B=2, S=512, Hq=8, Hkv=4, D=128, G=1)),
+])
+def test_attn_bwd_matches_oracle(basp, name, w):
+    got, ref = run_attn_bwd(basp, w)
+    for g, r, n in zip(got, ref, ("dQ", "dK", "dV")):
+        assert np.isfinite(g).all(), f"{name} {n}: not fully written"
+        assert_grad_close(g, r, f"{name} {n}")
+
+
+def test_attn_bwd_noncausal(basp):
+    w = synth.Workload("nc", N=2, B=2, S=256, Hq=2, Hkv=1, D=128)
+    got, ref = run_attn_bwd(basp, w, causal=False, seed=3)
+    for g, r, n in zip(got, ref, ("dQ", "dK", "dV")):
+        assert_grad_close(g, r, f"noncausal {n}")
+
+
+def test_layer_bwd_with_gradient_reshards(basp):
+    """Forward through basp_layer_fwd, backward through basp_layer_bwd on the saved head-sharded
+    activations, gradients back in the sequence-sharded layout; against the oracle's layer backward."""
+    w = synth.shrink(synth.WORKLOADS["llama3_8b_128k_train"], 256)
+    (Xq, Xk, Xv, Xdo), op = inputs(w, seed=1)
+    ref = oracle.layer_bwd(Xq, Xk, Xv, Xdo, op)
+    pl = make_plan(basp, w)
+    qs, ks, vs, dos = (to_dev(oracle.partition(X, op)) for X in (Xq, Xk, Xv, Xdo))
+    o = [torch.zeros_like(t) for t in qs]
+    lse = [torch.zeros((op.Bl, pl.Hq_l, w.S), dtype=torch.float32, device="cuda") for _ in range(w.N)]
+    ws = torch.empty(basp.basp_workspace_bytes(pl), dtype=torch.uint8, device="cuda")
+    basp.basp_clear_status()
+    basp.basp_layer_fwd(pl, qs, ks, vs, o, ws, lse)
+    qh, kh, vh, oh = (basp.as_shards(a) for a in basp.basp_layer_workspace_shards(pl, ws))
+    gq = [torch.full_like(t, float("nan")) for t in qs]
+    gk = [torch.full_like(t, float("nan")) for t in ks]
+    gv = [torch.full_like(t, float("nan")) for t in ks]
+    ws2 = torch.empty(basp.basp_layer_bwd_workspace_bytes(pl), dtype=torch.uint8, device="cuda")
+    basp.basp_layer_bwd(pl, qh, kh, vh, oh, lse, dos, gq, gk, gv, ws2)
+    basp.basp_get_status()
+    for g, n in ((gq, "dq_seq"), (gk, "dk_seq"), (gv, "dv_seq")):
+        assert_grad_close(to_f64(g), ref[n], n)
+
+
+def test_grads_reshard_single_launch_bit_exact(basp):
+    N, B, S, Hq, Hkv, D = 8, 2, 1024, 32, 8, 128
+    pl = basp.basp_plan_create(N, B, S, Hq, Hkv, D)
+    op = oracle.plan(N, B, S)
+    heads = [synth.random_bits((N, 1, S, h // op.K, D), seed=i) for i, h in enumerate((Hq, Hkv, Hkv))]
+    want = [oracle.h2s(a, op) for a in heads]
+    src = [to_dev(a) for a in heads]
+    dst = [[torch.zeros(x.shape[1:], dtype=torch.bfloat16, device="cuda") for _ in range(N)] for x in want]
+    n0 = basp.basp_launch_count()
+    basp.basp_reshard_grads_h2s(pl, *src, *dst)
+    torch.cuda.synchronize()
+    assert basp.basp_launch_count() == n0 + 1
+    for d, x in zip(dst, want):
+        assert np.array_equal(np.stack([synth.bits(t.cpu()) for t in d]), x)
