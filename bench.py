@@ -184,19 +184,40 @@ def run_gpu(args, w: synth.Workload):
     v_head = [torch.empty((Bl, w.S, plan.Hkv_l, w.D), dtype=torch.bfloat16, device=dev) for _ in range(N)]
     o_head = [torch.empty_like(t) for t in q_head]
 
+    train = w.train
+    if train:
+        do_seq = [randn((Bl, T, w.Hq, w.D)) for _ in range(N)]
+        do_head = [torch.empty_like(t) for t in q_head]
+        dq_head = [torch.empty_like(t) for t in q_head]
+        dk_head = [torch.empty_like(t) for t in k_head]
+        dv_head = [torch.empty_like(t) for t in k_head]
+        dq_seq = [torch.empty_like(t) for t in q_seq]
+        dk_seq = [torch.empty_like(t) for t in k_seq]
+        dv_seq = [torch.empty_like(t) for t in k_seq]
+        lse = [torch.empty((Bl, plan.Hq_l, w.S), dtype=torch.float32, device=dev) for _ in range(N)]
+        bwd_ws = torch.empty(basp.basp_attn_bwd_workspace_bytes(plan), dtype=torch.uint8, device=dev)
+    n_ev = 7 if train else 4
+
     def step(events=None):
-        """a2 -> a3 -> a4 (what basp_layer_fwd launches), with optional events between the launches."""
-        if events:
-            events[0].record()
+        """a2 -> a3 -> a4 (what basp_layer_fwd launches) and, for a training workload, a7 -> a6 -> a7
+        (what basp_layer_bwd launches), with optional events between the launches."""
+        def mark(i):
+            if events:
+                events[i].record()
+        mark(0)
         basp.basp_reshard_qkv_s2h(plan, q_seq, k_seq, v_seq, q_head, k_head, v_head)
-        if events:
-            events[1].record()
-        basp.basp_attn_fwd(plan, q_head, k_head, v_head, o_head)
-        if events:
-            events[2].record()
+        mark(1)
+        basp.basp_attn_fwd(plan, q_head, k_head, v_head, o_head, lse if train else None)
+        mark(2)
         basp.basp_reshard_h2s(plan, w.Hq, o_head, o_seq)
-        if events:
-            events[3].record()
+        mark(3)
+        if train:
+            basp.basp_reshard_s2h(plan, w.Hq, do_seq, do_head)
+            mark(4)
+            basp.basp_attn_bwd(plan, q_head, k_head, v_head, o_head, do_head, lse, dq_head, dk_head, dv_head, bwd_ws)
+            mark(5)
+            basp.basp_reshard_grads_h2s(plan, dq_head, dk_head, dv_head, dq_seq, dk_seq, dv_seq)
+            mark(6)
 
     basp.basp_clear_status()
     for _ in range(args.warmup):
@@ -204,7 +225,7 @@ def run_gpu(args, w: synth.Workload):
     torch.cuda.synchronize()
     basp.basp_get_status()
 
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(n_ev)] for _ in range(args.steps)]
     sampler = ClockSampler(local_rank) if rank == 0 else None
     launches0 = basp.basp_launch_count()
     pdist.barrier()
@@ -214,10 +235,11 @@ def run_gpu(args, w: synth.Workload):
     torch.cuda.synchronize()
     pdist.barrier()
     launches = basp.basp_launch_count() - launches0
-    total_ms = ev[0][0].elapsed_time(ev[-1][3])
+    total_ms = ev[0][0].elapsed_time(ev[-1][n_ev - 1])
     ms_s2h = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
     ms_attn = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
     ms_h2s = statistics.mean(e[2].elapsed_time(e[3]) for e in ev)
+    ms_bwd = [statistics.mean(e[i].elapsed_time(e[i + 1]) for e in ev) for i in (3, 4, 5)] if train else None
     basp.basp_get_status()
 
     if args.quick:     # kernel timings only (what the ncu recipes in profiles/ run)
@@ -225,9 +247,14 @@ def run_gpu(args, w: synth.Workload):
         if rank == 0:
             print(json.dumps({"workload": w.name, "ms_per_step": total_ms / args.steps, "ms_s2h": ms_s2h,
                               "ms_attn": ms_attn, "ms_h2s": ms_h2s, "gpu_launches": launches,
-                              "attn_tflops": w.attn_flops_fwd() / ms_attn / 1e9, "clocks": clocks}), flush=True)
+                              "attn_tflops": w.attn_flops_fwd() / ms_attn / 1e9, "clocks": clocks,
+                              "bwd_ms_s2h_attn_h2s": ms_bwd,
+                              "attn_bwd_tflops": (w.attn_flops_bwd() / ms_bwd[1] / 1e9) if train else None}), flush=True)
         pdist.finalize()
         return
+
+    if train:
+        return finish_train(args, w, basp, peaks, rank, world, sampler, launches, total_ms, ms_s2h, ms_attn, ms_h2s, ms_bwd, K)
 
     # fused layer (a5): one kernel straight from / to the sequence-sharded shards
     for _ in range(max(1, args.warmup // 2)):
@@ -305,6 +332,53 @@ def run_gpu(args, w: synth.Workload):
             },
             "fused": {"ms_per_step": ms_fused_max, "value": tokens_all / (ms_fused_max * 1e-3), "unit": UNIT,
                       "tflops": flops / (ms_fused * 1e-3) / 1e12, "launches_per_step": 1},
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    pdist.finalize()
+
+
+def finish_train(args, w, basp, peaks, rank, world, sampler, launches, total_ms, ms_s2h, ms_attn, ms_h2s, ms_bwd, K):
+    """JSON line of a forward + backward workload (BASELINE config 5)."""
+    clocks = sampler.stop() if sampler else None
+    ms_per_step = pdist.max_over_ranks(total_ms / args.steps)
+    tokens_all = w.tokens * world
+    if rank == 0:
+        fwd_tf = w.attn_flops_fwd() / (ms_attn * 1e-3) / 1e12
+        bwd_tf = w.attn_flops_bwd() / (ms_bwd[1] * 1e-3) / 1e12
+        gbs = lambda b, ms: b / (ms * 1e-3) / 1e9
+        cpu = None
+        if world == 1:
+            v, cores, desc, _ = oracle_sample(w, budget_rows=2048)
+            cpu = {"value": v / 3.5, "unit": UNIT, "cores": cores, "kind": "oracle",
+                   "sample": desc + "; forward sample scaled by 3.5 for forward + backward (4*D + 10*D flop per pair)"}
+        line = {
+            "metric": METRIC, "value": tokens_all / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "N": w.N, "b": w.B, "group_size": K, "S": w.S, "Hq": w.Hq, "Hkv": w.Hkv,
+                       "D": w.D, "causal": True,
+                       "path": "forward (s2h, attn_fwd, h2s) + backward (s2h dO, attn_bwd, h2s dQ/dK/dV)",
+                       "l2": "inputs larger than L2", "per_gpu_tokens": w.tokens},
+            "clocks": clocks, "e2e": None, "gpu_launches": launches,
+            "roofline": {"kernel": "attn_bwd (memset + Delta + main + dQ conversion)", "bound": "tensor",
+                         "achieved": bwd_tf, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
+                         "frac": bwd_tf / peaks["bf16_sustained"], "traffic": None,
+                         "peak_source": f"bf16 sustained, of {peaks['source']}", "ms": ms_bwd[1],
+                         "frac_of_burst": bwd_tf / peaks["bf16_burst"], "frac_of_nominal_2250": bwd_tf / 2250.0,
+                         "flops_per_launch": w.attn_flops_bwd()},
+            "kernels": {
+                "attn_fwd": {"ms": ms_attn, "bound": "tensor", "achieved": fwd_tf, "unit": "TFLOP/s",
+                             "frac": fwd_tf / peaks["bf16_sustained"]},
+                "reshard_qkv_s2h": {"ms": ms_s2h, "achieved": gbs(w.reshard_bytes_s2h(), ms_s2h), "unit": "GB/s",
+                                    "frac": gbs(w.reshard_bytes_s2h(), ms_s2h) / peaks["hbm_gbs"]},
+                "reshard_h2s_o": {"ms": ms_h2s, "achieved": gbs(w.reshard_bytes_h2s(), ms_h2s), "unit": "GB/s",
+                                  "frac": gbs(w.reshard_bytes_h2s(), ms_h2s) / peaks["hbm_gbs"]},
+                "reshard_s2h_do": {"ms": ms_bwd[0], "achieved": gbs(w.reshard_bytes_h2s(), ms_bwd[0]), "unit": "GB/s",
+                                   "frac": gbs(w.reshard_bytes_h2s(), ms_bwd[0]) / peaks["hbm_gbs"]},
+                "reshard_grads_h2s": {"ms": ms_bwd[2], "achieved": gbs(w.reshard_bytes_s2h(), ms_bwd[2]), "unit": "GB/s",
+                                      "frac": gbs(w.reshard_bytes_s2h(), ms_bwd[2]) / peaks["hbm_gbs"]},
+            },
             "cpu_baseline": cpu,
         }
         print(json.dumps(line), flush=True)

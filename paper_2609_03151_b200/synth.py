@@ -23,6 +23,7 @@ class Workload:
     Hkv: int
     D: int
     G: int = 0      # 0 -> BASP (G = B); 1 -> standard Ulysses
+    train: bool = False   # forward + backward step
 
     @property
     def K(self) -> int:
@@ -35,6 +36,10 @@ class Workload:
     def attn_flops_fwd(self) -> float:
         """4*D flop per unmasked (i,j) pair, S(S+1)/2 pairs per (sequence, q head)."""
         return 4.0 * self.D * (self.S * (self.S + 1) / 2) * self.B * self.Hq
+
+    def attn_flops_bwd(self) -> float:
+        """10*D flop per unmasked pair (five products, the recomputed scores included)."""
+        return 2.5 * self.attn_flops_fwd()
 
     def reshard_bytes_s2h(self) -> int:
         """Q, K and V each read once and written once."""
@@ -52,13 +57,13 @@ WORKLOADS = {
     "sweep_b4": Workload("sweep_b4", N=8, B=4, S=16384, Hq=32, Hkv=8, D=128),
     "sweep_b8": Workload("sweep_b8", N=8, B=8, S=8192, Hq=32, Hkv=8, D=128),
     "qwen25_7b_64k": Workload("qwen25_7b_64k", N=8, B=2, S=65536, Hq=28, Hkv=4, D=128),
-    "llama3_8b_128k_train": Workload("llama3_8b_128k_train", N=8, B=1, S=131072, Hq=32, Hkv=8, D=128),
+    "llama3_8b_128k_train": Workload("llama3_8b_128k_train", N=8, B=1, S=131072, Hq=32, Hkv=8, D=128, train=True),
 }
 
 
 def shrink(w: Workload, T: int = 512, name: str | None = None) -> Workload:
     """Same rank/head structure with T tokens per rank (S = T*K)."""
-    return Workload(name or f"{w.name}_T{T}", w.N, w.B, T * w.K, w.Hq, w.Hkv, w.D, w.G)
+    return Workload(name or f"{w.name}_T{T}", w.N, w.B, T * w.K, w.Hq, w.Hkv, w.D, w.G, w.train)
 
 
 def randn_bf16(gen: torch.Generator, shape) -> torch.Tensor:

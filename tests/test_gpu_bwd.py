@@ -106,3 +106,47 @@ def test_grads_reshard_single_launch_bit_exact(basp):
     assert basp.basp_launch_count() == n0 + 1
     for d, x in zip(dst, want):
         assert np.array_equal(np.stack([synth.bits(t.cpu()) for t in d]), x)
+
+
+def test_full_size_train_step_sampled(basp):
+    """BASELINE config 5 at full size (Llama-3-8B shape, N=8, b=1, S=131072), forward + backward:
+    sampled O and dQ rows anywhere in the sequence and dK/dV of the last 165 key positions (one full
+    tile and a ragged part of the previous one) against oracle rows / columns computed one by one."""
+    w = synth.WORKLOADS["llama3_8b_128k_train"]
+    q, k, v, do = synth.make_qkv(w, seed=0, with_dO=True)
+    pl = make_plan(basp, w)
+    Hl, Hkl = pl.Hq_l, pl.Hkv_l
+
+    def head_shards(x, hl):     # rank r of the single group owns heads [r*hl, (r+1)*hl) of the whole sequence
+        return [x[:, :, r * hl:(r + 1) * hl].contiguous().cuda() for r in range(w.N)]
+
+    dq_, dk_, dv_, ddo = head_shards(q, Hl), head_shards(k, Hkl), head_shards(v, Hkl), head_shards(do, Hl)
+    o = [torch.empty_like(t) for t in dq_]
+    lse = [torch.empty((1, Hl, w.S), dtype=torch.float32, device="cuda") for _ in range(w.N)]
+    gq = [torch.empty_like(t) for t in dq_]
+    gk = [torch.empty_like(t) for t in dk_]
+    gv = [torch.empty_like(t) for t in dk_]
+    ws = torch.empty(basp.basp_attn_bwd_workspace_bytes(pl), dtype=torch.uint8, device="cuda")
+    basp.basp_clear_status()
+    basp.basp_attn_fwd(pl, dq_, dk_, dv_, o, lse)
+    basp.basp_attn_bwd(pl, dq_, dk_, dv_, o, ddo, lse, gq, gk, gv, ws)
+    basp.basp_get_status()
+
+    Q, K, V, DO = (synth.bits(t) for t in (q, k, v, do))
+    rng = np.random.default_rng(0)
+    pos = [0, 1, 127, 128, 255, 256, 16383, 16384, 65535, 65536, w.S - 129, w.S - 128, w.S - 1]
+    pos += [int(x) for x in rng.integers(0, w.S, 11)]
+    rows = np.array([(0, h, i) for h in (0, 13, 31) for i in pos], dtype=np.int32)
+    ref_o, _ = oracle.attn_fwd_rows(Q, K, V, rows)
+    ref_dq = oracle.attn_bwd_dq_rows(Q, K, V, DO, rows)
+    got_o = np.stack([o[h // Hl][0, i, h % Hl].float().cpu().numpy().astype(np.float64) for _, h, i in rows])
+    got_dq = np.stack([gq[h // Hl][0, i, h % Hl].float().cpu().numpy().astype(np.float64) for _, h, i in rows])
+    err = np.abs(got_o - ref_o)
+    assert err.max() <= 2e-2 and err.mean() <= 2e-3, (err.max(), err.mean())
+    assert_grad_close(got_dq, ref_dq, "config 5 dQ rows")
+    ncols, kvh = 165, 3
+    ref_dk, ref_dv = oracle.attn_bwd_dkdv_tail(Q, K, V, DO, b=0, kv=kvh, ncols=ncols)
+    got_dk = gk[kvh // Hkl][0, w.S - ncols:, kvh % Hkl].float().cpu().numpy().astype(np.float64)
+    got_dv = gv[kvh // Hkl][0, w.S - ncols:, kvh % Hkl].float().cpu().numpy().astype(np.float64)
+    assert_grad_close(got_dk, ref_dk, "config 5 dK tail")
+    assert_grad_close(got_dv, ref_dv, "config 5 dV tail")
