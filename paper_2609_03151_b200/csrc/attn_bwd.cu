@@ -15,7 +15,8 @@
 //   (3) dV  += P^T dO       TS   -> TMEM [384,512)
 //   (4) dK  += dS^T Q       SS   -> TMEM [256,384)
 //   (5) dQ_m = dS K         SS   -> TMEM [128,256)  (A = the dS^T buffer read MN-major)
-//   compute warps: dQ_m added to the fp32 accumulator in global memory (red.add, order not fixed).
+//   compute warps: dQ_m staged through the (now free) Q / dO stage and added to the fp32 accumulator in
+//   global memory by TMA reduce-add (order of the additions not fixed).
 // Helper kernels: Delta = rowsum(dO * O); fp32 dQ accumulator -> bf16.
 #include <cuda.h>
 #include <math.h>
@@ -31,14 +32,15 @@ namespace {
 using namespace ptx;
 
 constexpr int kT = 128;
-constexpr int kBwdThreads = 320;          // 8 compute warps + TMA warp + MMA warp
+constexpr int kBwdComputeWarps = 16;
+constexpr int kBwdThreads = (kBwdComputeWarps + 2) * 32;   // compute warps + TMA warp + MMA warp
 
 template <int R>
 struct BwdParams {
     CUtensorMap q[R], k[R], v[R], dout[R];
+    CUtensorMap dq_acc[R];      // fp32 accumulator, box 32 floats x 1 head x 32 rows (reduce-add target)
     const float *lse[R];
     const float *delta[R];
-    float *dq_acc[R];
     __nv_bfloat16 *dk[R], *dv[R];
     int n_ranks, Bl, S, Hq_l, Hkv_l, q_per_kv, causal;
     float scale, scale_log2;
@@ -69,7 +71,7 @@ __device__ __forceinline__ bool bwd_get_item(const BwdParams<R> &p, int round, B
 }
 
 struct BwdBars {
-    uint64_t kv_full, kv_empty, qdo_full[2], qdo_empty[2];
+    uint64_t kv_full, kv_empty, qdo_full[2], qdo_empty[2], qdo_mma_done[2];
     uint64_t s_full, stats_full, pds_ready, dq_full, dq_read, dkdv_full, dkdv_read;
     uint32_t tmem_base;
     int abort_flag;
@@ -83,6 +85,15 @@ __device__ __forceinline__ void bwd_report(int *status, int code, int role, int 
     }
 }
 
+#ifdef BASP_PHASE_TIMING
+__device__ long long g_bwd_phase[32];
+#define BPH_T(var) const long long var = clock64()
+#define BPH_ADD(slot, a, b) do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (warp == 0 || warp == kBwdComputeWarps + 1)) g_bwd_phase[slot] += (b) - (a); } while (0)
+#else
+#define BPH_T(var)
+#define BPH_ADD(slot, a, b)
+#endif
+
 #define BWD_WAIT(bar, parity, role, detail)                                    \
     do {                                                                        \
         if (!mbar_wait((bar), (parity), &bars->abort_flag)) {                  \
@@ -91,11 +102,6 @@ __device__ __forceinline__ void bwd_report(int *status, int code, int role, int 
             goto bwd_done;                                                      \
         }                                                                       \
     } while (0)
-
-__device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float c, float d) {
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
-                 : "memory");
-}
 
 template <int R>
 __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_constant__ BwdParams<R> p) {
@@ -115,19 +121,23 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
 
     if (tid == 0) {
         mbar_init(&bars->kv_full, 1); mbar_init(&bars->kv_empty, 1);
-        for (int s = 0; s < 2; ++s) { mbar_init(&bars->qdo_full[s], 1); mbar_init(&bars->qdo_empty[s], 1); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&bars->qdo_full[s], 1);
+            mbar_init(&bars->qdo_empty[s], kBwdComputeWarps);   // every compute warp has drained its dQ block
+            mbar_init(&bars->qdo_mma_done[s], 1);
+        }
         mbar_init(&bars->s_full, 1);
-        mbar_init(&bars->stats_full, 8);
-        mbar_init(&bars->pds_ready, 8);
+        mbar_init(&bars->stats_full, kBwdComputeWarps);
+        mbar_init(&bars->pds_ready, kBwdComputeWarps);
         mbar_init(&bars->dq_full, 1);
-        mbar_init(&bars->dq_read, 8);
+        mbar_init(&bars->dq_read, kBwdComputeWarps);
         mbar_init(&bars->dkdv_full, 1);
-        mbar_init(&bars->dkdv_read, 8);
+        mbar_init(&bars->dkdv_read, kBwdComputeWarps);
         bars->abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         if (bars->abort_flag) bwd_report(p.status, 4, 0, (int)(smem_u32(smem) & 1023u));
         fence_mbar_init();
     }
-    if (warp == 8) { tmem_alloc(&bars->tmem_base, 512); tmem_relinquish(); }
+    if (warp == kBwdComputeWarps) { tmem_alloc(&bars->tmem_base, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -135,9 +145,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     constexpr uint32_t kColST = 0, kColDP = 128, kColDK = 256, kColDV = 384;
     if (bars->abort_flag) goto bwd_done;
 
-    if (warp < 8) {
+    if (warp < kBwdComputeWarps) {
         // ======================================================================= compute warps
-        const int w = warp >> 2;                        // which 64-column half of the score tile
+        const int g = warp >> 2;                        // which 32-column quarter of the score tile
         const int row = tid & 127;                      // TMEM lane: key row (scores) / query row (dQ)
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         uint32_t it_g = 0, item_n = 0;
@@ -149,44 +159,50 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     const int buf = it_g & 1;
                     {   // row statistics of the query tile: LSE (in log2 units) and Delta
                         const size_t off = ((size_t)item.bl * p.Hq_l + h) * p.S + (size_t)m * kT + row;
-                        if (w == 0) s_lse[buf * kT + row] = p.lse[item.r][off] * 1.4426950408889634f;
-                        else s_delta[buf * kT + row] = p.delta[item.r][off];
+                        if (g == 0) s_lse[buf * kT + row] = p.lse[item.r][off] * 1.4426950408889634f;
+                        else if (g == 1) s_delta[buf * kT + row] = p.delta[item.r][off];
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&bars->stats_full);
                     }
+                    BPH_T(t0);
                     BWD_WAIT(&bars->stats_full, it_g & 1, 10, m);
                     BWD_WAIT(&bars->s_full, it_g & 1, 11, m);
                     tc_fence_after();
-                    uint32_t st[64], dp[64];
-                    tmem_ld_x32(tmem + kColST + 64 * w + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&st[0]));
-                    tmem_ld_x32(tmem + kColST + 64 * w + 32 + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&st[32]));
-                    tmem_ld_x32(tmem + kColDP + 64 * w + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&dp[0]));
-                    tmem_ld_x32(tmem + kColDP + 64 * w + 32 + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&dp[32]));
+                    BPH_T(t1);
+                    uint32_t st[32], dp[32];
+                    tmem_ld_x32(tmem + kColST + 32 * g + lane_addr, st);
+                    tmem_ld_x32(tmem + kColDP + 32 * g + lane_addr, dp);
                     tmem_wait_ld();
+                    BPH_T(t2);
                     const bool diag = p.causal && m == item.n;
-                    const float *lse_b = s_lse + buf * kT + 64 * w;
-                    const float *del_b = s_delta + buf * kT + 64 * w;
+                    const float *lse_b = s_lse + buf * kT + 32 * g;
+                    const float *del_b = s_delta + buf * kT + 32 * g;
 #pragma unroll
-                    for (int c = 0; c < 64; c += 2) {
-                        float p0 = exp2_approx(fmaf(__uint_as_float(st[c]), p.scale_log2, -lse_b[c]));
-                        float p1 = exp2_approx(fmaf(__uint_as_float(st[c + 1]), p.scale_log2, -lse_b[c + 1]));
-                        if (diag) {                      // query 64w+c sees key `row` iff it is not earlier
-                            if (64 * w + c < row) p0 = 0.f;
-                            if (64 * w + c + 1 < row) p1 = 0.f;
+                    for (int c = 0; c < 32; c += 4) {
+                        const float4 l4 = *reinterpret_cast<const float4 *>(lse_b + c);
+                        const float4 d4 = *reinterpret_cast<const float4 *>(del_b + c);
+                        const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dl[4] = {d4.x, d4.y, d4.z, d4.w};
+                        float pv[4], dsv[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            pv[e] = exp2_approx(fmaf(__uint_as_float(st[c + e]), p.scale_log2, -lv[e]));
+                            if (diag && 32 * g + c + e < row) pv[e] = 0.f;   // query 32g+c+e is earlier than key `row`
+                            dsv[e] = pv[e] * (__uint_as_float(dp[c + e]) - dl[e]) * p.scale;
                         }
-                        const float d0 = p0 * (__uint_as_float(dp[c]) - del_b[c]) * p.scale;
-                        const float d1 = p1 * (__uint_as_float(dp[c + 1]) - del_b[c + 1]) * p.scale;
-                        st[c >> 1] = pack_bf16x2(p0, p1);
-                        dp[c >> 1] = pack_bf16x2(d0, d1);
+                        st[c >> 1] = pack_bf16x2(pv[0], pv[1]);
+                        st[(c >> 1) + 1] = pack_bf16x2(pv[2], pv[3]);
+                        dp[c >> 1] = pack_bf16x2(dsv[0], dsv[1]);
+                        dp[(c >> 1) + 1] = pack_bf16x2(dsv[2], dsv[3]);
                     }
-                    // P^T (bf16) over this half's own score columns: TMEM columns 64w .. 64w+31
-                    tmem_st_x32(tmem + kColST + 64 * w + lane_addr, *reinterpret_cast<const uint32_t(*)[32]>(&st[0]));
-                    // dS^T row `row`, query columns 64w..64w+63 = one 128-byte line of slab w (128-byte swizzle)
+                    BPH_T(t3);
+                    // P^T (bf16) over this quarter's own score columns: TMEM columns 32g .. 32g+15
+                    tmem_st_x16(tmem + kColST + 32 * g + lane_addr, *reinterpret_cast<const uint32_t(*)[16]>(&st[0]));
+                    // dS^T row `row`, query columns 32g..32g+31 = half a 128-byte line of slab g/2 (128-byte swizzle)
                     {
-                        uint8_t *line = sdS + w * 16384 + row * 128;
+                        uint8_t *line = sdS + (g >> 1) * 16384 + row * 128;
 #pragma unroll
-                        for (int ch = 0; ch < 8; ++ch)
-                            *reinterpret_cast<uint4 *>(line + ((ch ^ (row & 7)) << 4)) =
+                        for (int ch = 0; ch < 4; ++ch)
+                            *reinterpret_cast<uint4 *>(line + (((4 * (g & 1) + ch) ^ (row & 7)) << 4)) =
                                 make_uint4(dp[4 * ch], dp[4 * ch + 1], dp[4 * ch + 2], dp[4 * ch + 3]);
                     }
                     fence_proxy_async_smem();
@@ -195,33 +211,58 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars->pds_ready);
 
-                    // dQ_m tile: lane = query row, this half owns head-dim columns 64w .. 64w+63
+                    // dQ_m tile: lane = query row, this quarter owns head-dim columns 32g .. 32g+31
+                    BPH_T(t4);
                     BWD_WAIT(&bars->dq_full, it_g & 1, 12, m);
                     tc_fence_after();
-                    uint32_t dq[64];
-                    tmem_ld_x32(tmem + kColDP + 64 * w + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&dq[0]));
-                    tmem_ld_x32(tmem + kColDP + 64 * w + 32 + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&dq[32]));
+                    BPH_T(t5);
+                    uint32_t dq[32];
+                    tmem_ld_x32(tmem + kColDP + 32 * g + lane_addr, dq);
                     tmem_wait_ld();
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars->dq_read);
-                    float *dst = p.dq_acc[item.r] +
-                                 (((size_t)item.bl * p.S + (size_t)m * kT + row) * p.Hq_l + h) * D + 64 * w;
+                    // dQ leaves through the Q / dO stage of this step: once products (3) and (4) have read it, the
+                    // stage is 64 KiB of free shared memory = the fp32 dQ tile.  Quarter g owns the 16 KiB chunk g
+                    // ([128 rows][32 floats], 128-byte swizzle); each warp adds its own 32 rows with one TMA
+                    // reduce-add and releases the stage to the producer when the copy has read shared memory.
+                    {
+                        const uint32_t stage = it_g & 1, ph = (it_g >> 1) & 1;
+                        BWD_WAIT(&bars->qdo_mma_done[stage], ph, 14, m);
+                        uint8_t *chunk = (g < 2 ? sQ : sdO) + stage * kTileBytes + (g & 1) * 16384;
+                        uint8_t *line = chunk + row * 128;
 #pragma unroll
-                    for (int c = 0; c < 64; c += 4)
-                        red_add_v4(dst + c, __uint_as_float(dq[c]), __uint_as_float(dq[c + 1]),
-                                   __uint_as_float(dq[c + 2]), __uint_as_float(dq[c + 3]));
+                        for (int ch = 0; ch < 8; ++ch)
+                            *reinterpret_cast<uint4 *>(line + ((ch ^ (row & 7)) << 4)) =
+                                make_uint4(dq[4 * ch], dq[4 * ch + 1], dq[4 * ch + 2], dq[4 * ch + 3]);
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+#ifndef BWD_NO_RED
+                            tma_reduce_add_3d(&p.dq_acc[item.r], chunk + (warp & 3) * 4096, 32 * g, h,
+                                              item.bl * p.S + m * kT + (warp & 3) * 32);
+                            tma_store_commit();
+                            tma_store_wait_read<0>();
+#endif
+                            mbar_arrive(&bars->qdo_empty[stage]);
+                        }
+                    }
+                    BPH_T(t6);
+                    BPH_ADD(0, t0, t1); BPH_ADD(1, t1, t2); BPH_ADD(2, t2, t3); BPH_ADD(3, t3, t4);
+                    BPH_ADD(4, t4, t5); BPH_ADD(5, t5, t6); BPH_ADD(6, t0, t0 + 1);
                 }
             }
             // ---- item done: dK_n (half 0) / dV_n (half 1) to global as bf16
             BWD_WAIT(&bars->dkdv_full, item_n & 1, 13, item.n);
             tc_fence_after();
             {
-                __nv_bfloat16 *base = (w == 0 ? p.dk[item.r] : p.dv[item.r]) +
-                                      (((size_t)item.bl * p.S + (size_t)item.n * kT + row) * p.Hkv_l + item.hkv) * D;
-                const uint32_t col0 = (w == 0 ? kColDK : kColDV);
+                // quarters 0,1 write the two 64-column halves of dK, quarters 2,3 those of dV
+                __nv_bfloat16 *base = (g < 2 ? p.dk[item.r] : p.dv[item.r]) +
+                                      (((size_t)item.bl * p.S + (size_t)item.n * kT + row) * p.Hkv_l + item.hkv) * D +
+                                      64 * (g & 1);
+                const uint32_t col0 = (g < 2 ? kColDK : kColDV) + 64 * (g & 1);
 #pragma unroll
-                for (int cc = 0; cc < D / 32; ++cc) {
+                for (int cc = 0; cc < 2; ++cc) {
                     uint32_t rr[32];
                     tmem_ld_x32(tmem + col0 + cc * 32 + lane_addr, rr);
                     tmem_wait_ld();
@@ -240,7 +281,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->dkdv_read);
         }
-    } else if (warp == 8) {
+    } else if (warp == kBwdComputeWarps) {
         // ======================================================================= TMA producer
         uint32_t it_g = 0, item_n = 0;
         BwdItem item;
@@ -270,7 +311,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 }
             }
         }
-    } else if (warp == 9) {
+    } else if (warp == kBwdComputeWarps + 1) {
         // ======================================================================= MMA issuer
         const uint32_t idesc_kk = make_idesc_bf16(kT, kT, false, false);     // (1) (2): both operands K-major
         const uint32_t idesc_kn = make_idesc_bf16(kT, D, false, true);       // (3) (4): B is MN-major
@@ -288,8 +329,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 for (int m = item.m0; m < item.n_qt; ++m, ++it_g) {
                     const uint32_t stage = it_g & 1, ph = (it_g >> 1) & 1;
                     const uint32_t q16 = aQ + stage * (kTileBytes >> 4), do16 = adO + stage * (kTileBytes >> 4);
+                    BPH_T(u0);
                     BWD_WAIT(&bars->qdo_full[stage], ph, 31, m);
                     tc_fence_after();
+                    BPH_T(u1);
                     if (lane == 0) {        // (1) S^T = K Q^T
 #pragma unroll
                         for (int kk = 0; kk < D / 16; ++kk) {
@@ -297,8 +340,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                             mma_ss(tmem + kColST, desc_k | (uint64_t)(aK + off), desc_k | (uint64_t)(q16 + off), idesc_kk, kk > 0);
                         }
                     }
+                    BPH_T(u2);
                     BWD_WAIT(&bars->dq_read, (it_g & 1) ^ 1, 32, m);          // previous dQ tile has left TMEM
                     tc_fence_after();
+                    BPH_T(u3);
                     if (lane == 0) {        // (2) dP^T = V dO^T
 #pragma unroll
                         for (int kk = 0; kk < D / 16; ++kk) {
@@ -307,16 +352,25 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                         }
                         tc_commit(&bars->s_full);
                     }
+                    BPH_T(u4);
                     BWD_WAIT(&bars->pds_ready, it_g & 1, 33, m);
+                    BPH_T(u5);
                     if (first) BWD_WAIT(&bars->dkdv_read, (item_n & 1) ^ 1, 34, item.n);
                     tc_fence_after();
                     if (lane == 0) {
                         const uint32_t acc0 = first ? 0u : 1u;
-                        // (3) dV += P^T dO : A = P^T in TMEM (query index along K: 8 columns per 16 queries,
-                        //     the second half of the queries starts at column 64), B = dO read MN-major
+                        // (5) dQ_m = dS K : A = the dS^T buffer read MN-major (query rows), B = K MN-major.  Issued
+                        //     first so that the compute warps can take dQ out of TMEM while (3) and (4) run.
 #pragma unroll
                         for (int kk = 0; kk < kT / 16; ++kk)
-                            mma_ts(tmem + kColDV, tmem + kColST + (kk / 4) * 64 + (kk % 4) * 8,
+                            mma_ss(tmem + kColDP, desc_mn | (uint64_t)(adS + kk * 128), desc_mn | (uint64_t)(aK + kk * 128),
+                                   idesc_nn, kk > 0);
+                        tc_commit(&bars->dq_full);
+                        // (3) dV += P^T dO : A = P^T in TMEM (query index along K: 8 columns per 16 queries,
+                        //     each quarter of 32 queries starts at its own column 32g), B = dO read MN-major
+#pragma unroll
+                        for (int kk = 0; kk < kT / 16; ++kk)
+                            mma_ts(tmem + kColDV, tmem + kColST + (kk / 2) * 32 + (kk % 2) * 8,
                                    desc_mn | (uint64_t)(do16 + kk * 128), idesc_kn, kk > 0 ? 1u : acc0);
                         // (4) dK += dS^T Q : A = dS^T from shared memory (K-major: query columns), B = Q MN-major
 #pragma unroll
@@ -325,15 +379,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                             mma_ss(tmem + kColDK, desc_k | (uint64_t)(adS + off), desc_mn | (uint64_t)(q16 + kk * 128),
                                    idesc_kn, kk > 0 ? 1u : acc0);
                         }
-                        // (5) dQ_m = dS K : A = the same buffer read MN-major (query rows), B = K MN-major
-#pragma unroll
-                        for (int kk = 0; kk < kT / 16; ++kk)
-                            mma_ss(tmem + kColDP, desc_mn | (uint64_t)(adS + kk * 128), desc_mn | (uint64_t)(aK + kk * 128),
-                                   idesc_nn, kk > 0);
-                        tc_commit(&bars->dq_full);
-                        tc_commit(&bars->qdo_empty[stage]);
+                        tc_commit(&bars->qdo_mma_done[stage]);
                     }
                     first = false;
+                    BPH_T(u6);
+                    BPH_ADD(8, u0, u1); BPH_ADD(9, u1, u2); BPH_ADD(10, u2, u3); BPH_ADD(11, u3, u4);
+                    BPH_ADD(12, u4, u5); BPH_ADD(13, u5, u6); BPH_ADD(14, u0, u0 + 1);
                 }
             }
             if (lane == 0) {
@@ -351,7 +402,7 @@ bwd_done:
         while (globaltimer_ns() - t0 < 200000ull) { }
         __syncthreads();
     }
-    if (warp == 8) tmem_dealloc(tmem, 512);
+    if (warp == kBwdComputeWarps) tmem_dealloc(tmem, 512);
 }
 
 #undef BWD_WAIT
@@ -414,7 +465,9 @@ int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, 
         if (rc == BASP_OK) rc = tmap::encode_rows_heads_d(&prm.dout[r], dout[r], rows, pl->Hq_l, pl->D, kT);
         if (rc != BASP_OK) return rc;
         prm.lse[r] = lse[r];
-        prm.dq_acc[r] = reinterpret_cast<float *>(reinterpret_cast<char *>(acc0) + (size_t)r * acc_b);
+        float *acc_r = reinterpret_cast<float *>(reinterpret_cast<char *>(acc0) + (size_t)r * acc_b);
+        rc = tmap::encode_f32_rows_heads_d(&prm.dq_acc[r], acc_r, rows, pl->Hq_l, pl->D, 32);
+        if (rc != BASP_OK) return rc;
         prm.delta[r] = reinterpret_cast<float *>(reinterpret_cast<char *>(del0) + (size_t)r * del_b);
         prm.dk[r] = (__nv_bfloat16 *)dk[r];
         prm.dv[r] = (__nv_bfloat16 *)dv[r];
@@ -447,13 +500,22 @@ int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, 
 
     const long long n8 = (long long)(acc_b / sizeof(float) / 8);
     for (int r = 0; r < pl->N; ++r)
-        bwd_dq_convert_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>(prm.dq_acc[r], (__nv_bfloat16 *)dq[r], n8);
+        bwd_dq_convert_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>(
+            reinterpret_cast<const float *>(reinterpret_cast<const char *>(acc0) + (size_t)r * acc_b), (__nv_bfloat16 *)dq[r], n8);
     BASP_CUDA_TRY(cudaGetLastError());
     basp_count_launch(1 + 2 * pl->N);
     return BASP_OK;
 }
 
 }  // namespace
+
+#ifdef BASP_PHASE_TIMING
+extern "C" int basp_debug_bwd_phases(long long *out, int reset) {
+    if (out && cudaMemcpyFromSymbol(out, g_bwd_phase, sizeof(long long) * 32) != cudaSuccess) return -1;
+    if (reset) { long long z[32] = {0}; if (cudaMemcpyToSymbol(g_bwd_phase, z, sizeof(z)) != cudaSuccess) return -1; }
+    return 0;
+}
+#endif
 
 extern "C" size_t basp_attn_bwd_workspace_bytes(const basp_plan *p) {
     if (!p) return 0;

@@ -83,6 +83,13 @@ __device__ __forceinline__ void tma_store_3d(const void *tmap, const void *smem_
         ::"l"(tmap), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
+// 3-D tiled reduce-add shared -> global (element type and swizzle come from the tensor map).
+__device__ __forceinline__ void tma_reduce_add_3d(const void *tmap, const void *smem_src, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+        ::"l"(tmap), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int kPending>
 __device__ __forceinline__ void tma_store_wait_read() {

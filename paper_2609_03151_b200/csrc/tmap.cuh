@@ -47,4 +47,27 @@ inline int encode_rows_heads_d(CUtensorMap *out, const void *base, uint64_t rows
     return BASP_OK;
 }
 
+// fp32 tensor [rows][heads][D] seen as 3-D (D, heads, rows); box = 32 x 1 x box_rows floats (128-byte
+// lines) with the 128-byte swizzle: the shape of one warp's share of an accumulator tile.
+inline int encode_f32_rows_heads_d(CUtensorMap *out, const void *base, uint64_t rows, uint64_t heads, uint64_t D,
+                                   uint32_t box_rows) {
+    EncodeTiledFn fn = encoder();
+    if (!fn) {
+        basp_set_cuda_error("cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)", -1, "driver entry point not found");
+        return BASP_ERR_CUDA;
+    }
+    cuuint64_t dims[3] = {D, heads, rows};
+    cuuint64_t strides[2] = {D * 4, heads * D * 4};
+    cuuint32_t box[3] = {32, 1, box_rows};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        basp_set_cuda_error("cuTensorMapEncodeTiled(f32)", (int)r, "tensor map encoding failed");
+        return BASP_ERR_CUDA;
+    }
+    return BASP_OK;
+}
+
 }  // namespace tmap
