@@ -213,9 +213,14 @@ size_t basp_layer_bwd_workspace_bytes(const basp_plan *plan);
 
 /* ---- the fused layer for callers whose shards are in HOST memory: copies every Q/K/V
  * shard host->device into `device_arena` (device memory, >= basp_host_arena_bytes(plan)
- * bytes), runs basp_layer_fwd_fused, copies every O shard device->host and waits for the
- * stream.  q/k/v/o_seq_host are host arrays of n_ranks HOST pointers (pinned memory makes
- * the copies asynchronous; pageable memory works, slower). */
+ * bytes), runs the fused kernel, copies every O shard device->host and waits for the stream.
+ * Copies and kernels are pipelined: with the causal mask the rows of local rank l need only the
+ * shards of local ranks 0..l of its group, so one launch per local rank starts as soon as that
+ * shard has arrived, and its O shard is read back while later ones are still computed.  The
+ * copies run on two library-owned streams (created on first use, per device; no device memory);
+ * calls that overlap in time on one device share them and must be serialised by the caller.
+ * q/k/v/o_seq_host are host arrays of n_ranks HOST pointers (pinned memory makes the copies
+ * asynchronous; pageable memory works, slower). */
 int basp_layer_fwd_host(const basp_plan *plan, const void *const *q_seq_host,
                         const void *const *k_seq_host, const void *const *v_seq_host,
                         void *const *o_seq_host, void *device_arena, size_t arena_bytes,

@@ -19,7 +19,9 @@ struct AttnParams {
     float *lse[R];
     int n_ranks, K, Bl, S, T, Hq_l, Hkv_l, q_per_kv;
     int o_heads;            // heads in one row of the O destination (Hq_l, or Hq when fused)
-    int qb_band;            // query blocks per scheduling band (divides the number of 256-row blocks)
+    int qb_band;            // query blocks per scheduling band (divides qb_count)
+    int r_begin, r_count;   // ranks covered by this launch
+    int qb_begin, qb_count; // 256-row query blocks covered by this launch
     int fused, causal, has_lse;
     float scale_log2;       // softmax scale * log2(e)
     int *status;

@@ -40,9 +40,8 @@ struct WsItem {
 template <int R>
 __device__ __forceinline__ bool ws_get_item(const AttnParams<R> &p, int round, WsItem &it) {
     const int n_qt = p.S / kTile;
-    const int n_qb = (n_qt + 1) / 2;
-    const int per_qb = p.n_ranks * p.Bl * p.Hq_l;
-    const int total = n_qb * per_qb;
+    const int per_qb = p.r_count * p.Bl * p.Hq_l;
+    const int total = p.qb_count * per_qb;
     const int pos = (round & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x;   // boustrophedon
     const int i = round * (int)gridDim.x + pos;
     if (i >= total) return false;
@@ -56,12 +55,12 @@ __device__ __forceinline__ bool ws_get_item(const AttnParams<R> &p, int round, W
     const int stream = rem / per_stream;
     rem -= stream * per_stream;
     const int qb_in_band = rem / p.q_per_kv;
-    it.qb = n_qb - 1 - (band * p.qb_band + qb_in_band);
+    it.qb = p.qb_begin + p.qb_count - 1 - (band * p.qb_band + qb_in_band);
     it.hkv = stream % p.Hkv_l;
     it.h = it.hkv * p.q_per_kv + (rem - qb_in_band * p.q_per_kv);
     const int sb = stream / p.Hkv_l;
     it.bl = sb % p.Bl;
-    it.r = sb / p.Bl;
+    it.r = p.r_begin + sb / p.Bl;
     const int qt0 = 2 * it.qb, qt1 = qt0 + 1;
     const bool has1 = qt1 < n_qt;
     it.n[0] = p.causal ? qt0 + 1 : n_qt;

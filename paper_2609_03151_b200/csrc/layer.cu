@@ -2,8 +2,13 @@
 // through a caller-provided workspace, and the host-buffer wrapper around the fused kernel.
 #include "common.cuh"
 
+#include <mutex>
+
 int basp_attn_dispatch(const basp_plan *pl, const void *const *q, const void *const *k, const void *const *v,
                        void *const *o, float *const *lse, float scale, bool fused, void *stream);
+int basp_attn_dispatch_range(const basp_plan *pl, const void *const *q, const void *const *k, const void *const *v,
+                             void *const *o, float *const *lse, float scale, bool fused, const int *range,
+                             void *stream);
 
 namespace {
 size_t q_shard_bytes(const basp_plan *p) { return (size_t)p->Bl * p->T * p->Hq * p->D * 2; }
@@ -85,6 +90,41 @@ extern "C" int basp_layer_bwd(const basp_plan *p, const void *const *q_head, con
     return basp_reshard_grads_h2s(p, dqh, dkh, dvh, dq_seq, dk_seq, dv_seq, stream);
 }
 
+namespace {
+// Copy streams and events of the host-buffer entry, created once per device (no device memory).
+struct HostPipe {
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, done = nullptr, arrived[BASP_MAX_RANKS] = {}, computed[BASP_MAX_RANKS] = {};
+};
+std::mutex g_pipe_mu;
+HostPipe g_pipes[64];
+
+int get_pipe(HostPipe **out) {
+    int dev = -1;
+    BASP_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return BASP_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_pipe_mu);
+    HostPipe &p = g_pipes[dev];
+    if (!p.in) {
+        BASP_CUDA_TRY(cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking));
+        BASP_CUDA_TRY(cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking));
+        BASP_CUDA_TRY(cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming));
+        BASP_CUDA_TRY(cudaEventCreateWithFlags(&p.done, cudaEventDisableTiming));
+        for (int i = 0; i < BASP_MAX_RANKS; ++i) {
+            BASP_CUDA_TRY(cudaEventCreateWithFlags(&p.arrived[i], cudaEventDisableTiming));
+            BASP_CUDA_TRY(cudaEventCreateWithFlags(&p.computed[i], cudaEventDisableTiming));
+        }
+    }
+    *out = &p;
+    return BASP_OK;
+}
+}  // namespace
+
+// Copies, kernels and read-backs are pipelined.  With the causal mask the query rows that local rank l
+// owns only need the shards of local ranks 0..l of its group, so the launch for those rows starts as soon
+// as shard l has arrived while later shards are still on the bus, and O shard l is read back as soon as
+// that launch is done (three streams: copies in, the caller's stream for the kernels, copies out).
+// Calls that overlap in time on one device share the internal streams and events: serialise them.
 extern "C" int basp_layer_fwd_host(const basp_plan *p, const void *const *q_seq_host, const void *const *k_seq_host,
                                    const void *const *v_seq_host, void *const *o_seq_host, void *device_arena,
                                    size_t arena_bytes, float softmax_scale, void *stream) {
@@ -92,6 +132,9 @@ extern "C" int basp_layer_fwd_host(const basp_plan *p, const void *const *q_seq_
     if (!aligned16(device_arena)) return BASP_ERR_ALIGN;
     if (arena_bytes < basp_host_arena_bytes(p)) return BASP_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    HostPipe *pipe = nullptr;
+    int rc = get_pipe(&pipe);
+    if (rc != BASP_OK) return rc;
     char *w = (char *)device_arena;
     void *qd[BASP_MAX_RANKS], *kd[BASP_MAX_RANKS], *vd[BASP_MAX_RANKS], *od[BASP_MAX_RANKS];
     const size_t qb = q_shard_bytes(p), kb = kv_shard_bytes(p);
@@ -101,14 +144,42 @@ extern "C" int basp_layer_fwd_host(const basp_plan *p, const void *const *q_seq_
         kd[r] = w + (size_t)p->N * qb + (size_t)r * kb;
         vd[r] = w + (size_t)p->N * (qb + kb) + (size_t)r * kb;
         od[r] = w + (size_t)p->N * (qb + 2 * kb) + (size_t)r * qb;
-        BASP_CUDA_TRY(cudaMemcpyAsync(qd[r], q_seq_host[r], qb, cudaMemcpyHostToDevice, st));
-        BASP_CUDA_TRY(cudaMemcpyAsync(kd[r], k_seq_host[r], kb, cudaMemcpyHostToDevice, st));
-        BASP_CUDA_TRY(cudaMemcpyAsync(vd[r], v_seq_host[r], kb, cudaMemcpyHostToDevice, st));
     }
-    int rc = basp_attn_dispatch(p, qd, kd, vd, od, nullptr, softmax_scale, true, stream);
-    if (rc != BASP_OK) return rc;
-    for (int r = 0; r < p->N; ++r)
-        BASP_CUDA_TRY(cudaMemcpyAsync(o_seq_host[r], od[r], qb, cudaMemcpyDeviceToHost, st));
+    const bool by_chunk = p->causal && p->T % 256 == 0;     // a launch per local rank's rows, else per group
+    BASP_CUDA_TRY(cudaEventRecord(pipe->start, st));
+    BASP_CUDA_TRY(cudaStreamWaitEvent(pipe->in, pipe->start, 0));
+    BASP_CUDA_TRY(cudaStreamWaitEvent(pipe->out, pipe->start, 0));
+    for (int r = 0; r < p->N; ++r) {
+        BASP_CUDA_TRY(cudaMemcpyAsync(kd[r], k_seq_host[r], kb, cudaMemcpyHostToDevice, pipe->in));
+        BASP_CUDA_TRY(cudaMemcpyAsync(vd[r], v_seq_host[r], kb, cudaMemcpyHostToDevice, pipe->in));
+        BASP_CUDA_TRY(cudaMemcpyAsync(qd[r], q_seq_host[r], qb, cudaMemcpyHostToDevice, pipe->in));
+        BASP_CUDA_TRY(cudaEventRecord(pipe->arrived[r], pipe->in));
+    }
+    for (int g = 0; g < p->G; ++g) {
+        const int r0 = g * p->K;
+        if (by_chunk) {
+            for (int l = 0; l < p->K; ++l) {
+                BASP_CUDA_TRY(cudaStreamWaitEvent(st, pipe->arrived[r0 + l], 0));
+                const int range[4] = {r0, p->K, l * (p->T / 256), p->T / 256};
+                rc = basp_attn_dispatch_range(p, qd, kd, vd, od, nullptr, softmax_scale, true, range, stream);
+                if (rc != BASP_OK) return rc;
+                BASP_CUDA_TRY(cudaEventRecord(pipe->computed[r0 + l], st));
+                BASP_CUDA_TRY(cudaStreamWaitEvent(pipe->out, pipe->computed[r0 + l], 0));
+                BASP_CUDA_TRY(cudaMemcpyAsync(o_seq_host[r0 + l], od[r0 + l], qb, cudaMemcpyDeviceToHost, pipe->out));
+            }
+        } else {
+            BASP_CUDA_TRY(cudaStreamWaitEvent(st, pipe->arrived[r0 + p->K - 1], 0));
+            const int range[4] = {r0, p->K, 0, (p->S / 128 + 1) / 2};
+            rc = basp_attn_dispatch_range(p, qd, kd, vd, od, nullptr, softmax_scale, true, range, stream);
+            if (rc != BASP_OK) return rc;
+            BASP_CUDA_TRY(cudaEventRecord(pipe->computed[r0], st));
+            BASP_CUDA_TRY(cudaStreamWaitEvent(pipe->out, pipe->computed[r0], 0));
+            for (int l = 0; l < p->K; ++l)
+                BASP_CUDA_TRY(cudaMemcpyAsync(o_seq_host[r0 + l], od[r0 + l], qb, cudaMemcpyDeviceToHost, pipe->out));
+        }
+    }
+    BASP_CUDA_TRY(cudaEventRecord(pipe->done, pipe->out));
+    BASP_CUDA_TRY(cudaStreamWaitEvent(st, pipe->done, 0));
     BASP_CUDA_TRY(cudaStreamSynchronize(st));
     return BASP_OK;
 }
