@@ -19,9 +19,6 @@
 int *basp_status_device_ptr();
 
 #ifdef BASP_PHASE_TIMING
-extern "C" int basp_debug_trace(long long *out) {
-    return cudaMemcpyFromSymbol(out, g_trace, sizeof(long long) * 4 * 256) == cudaSuccess ? 0 : -1;
-}
 extern "C" int basp_debug_phases(long long *out, int reset) {
     if (out && cudaMemcpyFromSymbol(out, g_phase_cycles, sizeof(long long) * 64) != cudaSuccess) return -1;
     if (reset) { long long z[64] = {0}; if (cudaMemcpyToSymbol(g_phase_cycles, z, sizeof(z)) != cudaSuccess) return -1; }

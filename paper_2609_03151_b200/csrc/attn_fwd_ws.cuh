@@ -84,14 +84,7 @@ __device__ long long g_phase_cycles[64];
 #define PHASE_T(var) const long long var = clock64()
 #define PHASE_ADD(slot, a, b) do { if (blockIdx.x == 0 && (threadIdx.x & 127) == 0) g_phase_cycles[slot] += (b) - (a); } while (0)
 #define PHASE_ADD1(slot, a, b) do { if (blockIdx.x == 0) g_phase_cycles[slot] += (b) - (a); } while (0)
-__device__ long long g_trace[4][256];
-// record (event id, clock) of iterations 200..205 of a role's leader thread in CTA 0
-#define TRACE(role, iter, ev) do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (iter) >= 200 && (iter) < 206 && tr_n < 127) { \
-    g_trace[role][2 * tr_n] = (ev) + 100 * (long long)(iter); g_trace[role][2 * tr_n + 1] = clock64(); ++tr_n; } } while (0)
-#define TRACE_DECL int tr_n = 0
 #else
-#define TRACE(role, iter, ev)
-#define TRACE_DECL
 #define PHASE_T(var)
 #define PHASE_ADD(slot, a, b)
 #define PHASE_ADD1(slot, a, b)
@@ -145,13 +138,12 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
 
     if (warp < 8) {
         // =============================================================== softmax of query tile t
-        reg_inc<176>();
+        reg_inc<192>();
         const int t = warp >> 2;
         const int row = tid & 127;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t S_t = tmem + 128 * t + lane_addr;
         uint32_t it_cnt = 0, ep_cnt = 0;
-        TRACE_DECL;
         WsItem item;
         for (int round = 0; ws_get_item(p, round, item); ++round) {
             const int n_t = item.n[t];
@@ -162,7 +154,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 WS_WAIT(&sh.s_full[t], it_cnt & 1, 10 + t, j);
                 tc_fence_after();
                 PHASE_T(c1);
-                if ((warp & 3) == 0) TRACE(t, it_cnt, 1);
                 uint32_t s[kTile];
                 tmem_ld_x32(S_t + 0, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
                 tmem_ld_x32(S_t + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
@@ -170,7 +161,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 tmem_ld_x32(S_t + 96, *reinterpret_cast<uint32_t(*)[32]>(&s[96]));
                 tmem_wait_ld();
                 PHASE_T(c2);
-                if ((warp & 3) == 0) TRACE(t, it_cnt, 2);
                 if (p.causal && j == n_t - 1) {        // diagonal tile: key column i visible iff i <= row
 #pragma unroll
                     for (int i = 0; i < kTile; ++i)
@@ -189,7 +179,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
                                  fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
                 mx *= p.scale_log2;
-                if ((warp & 3) == 0) TRACE(t, it_cnt, 3);
                 float m_new, alpha;
                 if (j == 0) { m_new = mx; alpha = 1.f; }
                 else if (mx > m_ref + kRescaleThreshold) { m_new = mx; alpha = exp2_approx(m_ref - m_new); }
@@ -199,7 +188,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 if (lane == 0) mbar_arrive(&sh.alpha_full[t]);
                 m_ref = m_new;
                 PHASE_T(c3);
-                if ((warp & 3) == 0) TRACE(t, it_cnt, 4);
                 const uint64_t sc2 = pack_f2(p.scale_log2, p.scale_log2), nm2 = pack_f2(-m_new, -m_new);
                 uint64_t rs2[2] = {0ull, 0ull};
                 auto exp_row = [&](auto diag_tag) {
@@ -230,7 +218,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 unpack_f2(add2(rs2[0], rs2[1]), ra, rb);
                 l_run = l_run * alpha + (ra + rb);
                 PHASE_T(c4);
-                if ((warp & 3) == 0) TRACE(t, it_cnt, 5);
                 tmem_st_x32(S_t + 0, *reinterpret_cast<const uint32_t(*)[32]>(&s[0]));
                 tmem_st_x32(S_t + 32, *reinterpret_cast<const uint32_t(*)[32]>(&s[32]));
                 tmem_wait_st();
@@ -238,7 +225,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.p_full[t]);
                 PHASE_T(c5);
-                if ((warp & 3) == 0) TRACE(t, it_cnt, 6);
                 PHASE_ADD(8 * t + 0, c0, c1); PHASE_ADD(8 * t + 1, c1, c2); PHASE_ADD(8 * t + 2, c2, c3);
                 PHASE_ADD(8 * t + 3, c3, c4); PHASE_ADD(8 * t + 4, c4, c5); PHASE_ADD(8 * t + 5, c0, c0 + 1);
             }
@@ -254,7 +240,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
         }
     } else if (warp < 12) {
         // =============================================================== correction + epilogue
-        reg_dec<80>();
+        reg_dec<64>();
         const int row = tid & 127;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         uint32_t it_cnt[2] = {0, 0}, ep_cnt[2] = {0, 0};
@@ -318,7 +304,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
             }
         }
     } else {
-        reg_dec<80>();
+        reg_dec<64>();
         if (warp == 12) {
             // =========================================================== TMA producer (lane 0 issues)
             uint32_t kv_it = 0, item_n = 0;
@@ -353,8 +339,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
             const uint32_t idesc_qk = make_idesc_bf16(kTile, kTile, false, false);
             const uint32_t idesc_pv = make_idesc_bf16(kTile, D, false, true);
             uint32_t kv_it = 0, item_n = 0, it_cnt[2] = {0, 0}, ep_cnt[2] = {0, 0};
-            TRACE_DECL;
-            WsItem item;
+                WsItem item;
             // Descriptors differ only in the 14-bit start-address field, so a step along K is an add.
             const uint64_t desc_k = make_smem_desc_sw128(0, 16, 1024);        // K-major operands (Q, K)
             const uint64_t desc_v = make_smem_desc_sw128(0, 16384, 1024);     // MN-major operand (V)
@@ -399,12 +384,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                             PHASE_T(d0);
                             if (j == 0) WS_WAIT(&sh.o_free[t], (ep_cnt[t] & 1) ^ 1, 43 + t, round);
                             PHASE_T(d1);
-                            TRACE(2, it_cnt[t], 10 + t);
                             WS_WAIT(&sh.p_full[t], it_cnt[t] & 1, 45 + t, j);
                             PHASE_T(d2);
                             WS_WAIT(&sh.o_rescaled[t], it_cnt[t] & 1, 47 + t, j);
                             PHASE_T(d3);
-                            TRACE(2, it_cnt[t], 20 + t);
                             ++it_cnt[t];
                             tc_fence_after();
                             const uint64_t b = desc_v | (uint64_t)(kv_addr16 + slot_v * (kTileBytes >> 4));
@@ -416,7 +399,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                             }
                             if (j == item.n[t] - 1) { commit(&sh.o_final[t]); ++ep_cnt[t]; }
                             PHASE_T(d4);
-                            TRACE(2, it_cnt[t] - 1, 30 + t);
                             PHASE_ADD1(16, d0, d1); PHASE_ADD1(17 + t, d1, d2); PHASE_ADD1(19, d2, d3); PHASE_ADD1(20, d3, d4);
                         }
                         if (t == last_v) commit(&sh.kv_empty[slot_v]);
@@ -431,7 +413,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                                 tc_fence_after();
                             }
                             issue_qk(t, slot_k);
-                            TRACE(2, it_cnt[t] - 1, 40 + t);
                             if (t == last_k) {
                                 commit(&sh.kv_empty[slot_k]);
                                 if (j + 2 == item.n_max) commit(&sh.q_empty);   // that was the item's last Q.K^T
