@@ -18,6 +18,10 @@
 
 int *basp_status_device_ptr();
 
+#ifndef BASP_BAND_TARGET
+#define BASP_BAND_TARGET 32   // CTAs that share one KV stream at a time (query blocks per band x query heads per KV head)
+#endif
+
 #ifdef BASP_PHASE_TIMING
 extern "C" int basp_debug_phases(long long *out, int reset) {
     if (out && cudaMemcpyFromSymbol(out, g_phase_cycles, sizeof(long long) * 64) != cudaSuccess) return -1;
@@ -48,7 +52,7 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
     {
         const int q_per_kv = pl->Hq / pl->Hkv;
         prm.r_begin = range[0]; prm.r_count = range[1]; prm.qb_begin = range[2]; prm.qb_count = range[3];
-        int band = 16 / q_per_kv < 1 ? 1 : (16 / q_per_kv > 8 ? 8 : 16 / q_per_kv);
+        int band = BASP_BAND_TARGET / q_per_kv < 1 ? 1 : (BASP_BAND_TARGET / q_per_kv > 16 ? 16 : BASP_BAND_TARGET / q_per_kv);
         while (prm.qb_count % band != 0) --band;
         prm.qb_band = band;
     }
