@@ -90,9 +90,13 @@ __device__ long long g_phase_cycles[64];
 #define PHASE_ADD1(slot, a, b)
 #endif
 
+#ifndef BASP_SLEEP_NS
+#define BASP_SLEEP_NS 32    // back-off of the correction and producer warps while they wait
+#endif
+
 #define WS_WAIT(bar, parity, role, detail)                                     \
     do {                                                                        \
-        if (!mbar_wait((bar), (parity), &sh.abort_flag)) {                     \
+        if (!mbar_wait((bar), (parity), &sh.abort_flag, ((role) >= 20 && (role) < 40) ? BASP_SLEEP_NS : 0)) { \
             sh.abort_flag = 1;                                                  \
             report(p.status, 1, (role), (detail));                              \
             goto ws_done;                                                       \
