@@ -127,7 +127,7 @@ int basp_reshard_qkv_s2h(const basp_plan *plan, const void *const *q_seq, const 
  * Inputs/outputs are HEAD-sharded; lse_shards may be NULL (then no LSE is written), else a
  * host array of n_ranks device pointers to fp32 [Bl][Hq/K][S].  softmax_scale = 0 selects
  * 1/sqrt(D).  bf16 operands, fp32 accumulation and softmax, P rounded to bf16 before P.V.
- * Requires D in {64, 128} and S a multiple of 128 (else BASP_ERR_UNSUPPORTED).
+ * Requires D in {64, 128} (else BASP_ERR_UNSUPPORTED); S is arbitrary (a ragged last tile is masked).
  * A bounded wait that expires inside the kernel is reported by basp_get_status. */
 int basp_attn_fwd(const basp_plan *plan, const void *const *q_head, const void *const *k_head,
                   const void *const *v_head, void *const *o_head, float *const *lse_shards,
@@ -167,7 +167,8 @@ int basp_layer_fwd_static(const basp_plan *plan, const void *const *q_seq, const
 /* ---- the same layer as ONE kernel: attention tiles are fetched straight from the
  * sequence-sharded sources (token tile at sequence position s lives on rank gK + s/T) and
  * O tiles are stored straight into the sequence-sharded destination, so the head-sharded
- * copies never exist.  Additionally requires T to be a multiple of 128.  No workspace. */
+ * copies never exist.  Requires T to be a multiple of 128 (a tile must not straddle two ranks), else
+ * BASP_ERR_UNSUPPORTED.  No workspace. */
 int basp_layer_fwd_fused(const basp_plan *plan, const void *const *q_seq, const void *const *k_seq,
                          const void *const *v_seq, void *const *o_seq, float *const *lse_shards,
                          float softmax_scale, void *stream);

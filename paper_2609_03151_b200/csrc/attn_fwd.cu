@@ -91,7 +91,7 @@ int basp_attn_dispatch_range(const basp_plan *pl, const void *const *q, const vo
                              void *const *o, float *const *lse, float scale, bool fused, const int *range,
                              void *stream) {
     if (!pl || !q || !k || !v || !o) return BASP_ERR_NULL;
-    if ((pl->D != 64 && pl->D != 128) || pl->S % kTile != 0) return BASP_ERR_UNSUPPORTED;
+    if (pl->D != 64 && pl->D != 128) return BASP_ERR_UNSUPPORTED;
     if (fused && pl->T % kTile != 0) return BASP_ERR_UNSUPPORTED;
     for (int r = 0; r < pl->N; ++r) {
         if (!q[r] || !k[r] || !v[r] || !o[r] || (lse && !lse[r])) return BASP_ERR_NULL;
@@ -100,7 +100,7 @@ int basp_attn_dispatch_range(const basp_plan *pl, const void *const *q, const vo
         for (int r2 = 0; r2 < pl->N; ++r2)
             if (o[r] == q[r2] || o[r] == k[r2] || o[r] == v[r2]) return BASP_ERR_ALIAS;
     }
-    const int full[4] = {0, pl->N, 0, (pl->S / kTile + 1) / 2};
+    const int full[4] = {0, pl->N, 0, ((pl->S + kTile - 1) / kTile + 1) / 2};
     if (!range) range = full;
     if (range[1] <= 0 || range[3] <= 0) return BASP_OK;
     if (pl->N <= 8) return fill_and_launch<8>(pl, q, k, v, o, lse, scale, fused, range, (cudaStream_t)stream);

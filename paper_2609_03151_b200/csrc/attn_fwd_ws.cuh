@@ -39,7 +39,7 @@ struct WsItem {
 
 template <int R>
 __device__ __forceinline__ bool ws_get_item(const AttnParams<R> &p, int round, WsItem &it) {
-    const int n_qt = p.S / kTile;
+    const int n_qt = (p.S + kTile - 1) / kTile;       // the last tile may be ragged
     const int per_qb = p.r_count * p.Bl * p.Hq_l;
     const int total = p.qb_count * per_qb;
     const int pos = (round & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x;   // boustrophedon
@@ -165,10 +165,17 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 tmem_ld_x32(S_t + 96, *reinterpret_cast<uint32_t(*)[32]>(&s[96]));
                 tmem_wait_ld();
                 PHASE_T(c2);
-                if (p.causal && j == n_t - 1) {        // diagonal tile: key column i visible iff i <= row
+                // Key column i of this tile is visible iff i <= lim: the causal diagonal (i <= row) and, in a
+                // ragged last tile, the end of the sequence (i < S - 128 j; what lies beyond belongs to the next
+                // sequence of the shard or is TMA zero fill).
+                int lim = kTile - 1;
+                if (p.causal && j == n_t - 1) lim = row;
+                if (p.S - j * kTile - 1 < lim) lim = p.S - j * kTile - 1;
+                const bool masked = __any_sync(0xffffffffu, lim < kTile - 1);
+                if (masked) {
 #pragma unroll
                     for (int i = 0; i < kTile; ++i)
-                        if (i > row) s[i] = 0xff800000u;   // -inf
+                        if (i > lim) s[i] = 0xff800000u;   // -inf
                 }
                 float mxs[8];
 #pragma unroll
@@ -209,14 +216,14 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                             e1 = exp2_approx(x1);
                         }
                         if (kDiag) {                  // masked keys contribute exactly nothing
-                            if (i > row) e0 = 0.f;
-                            if (i + 1 > row) e1 = 0.f;
+                            if (i > lim) e0 = 0.f;
+                            if (i + 1 > lim) e1 = 0.f;
                         }
                         rs2[(i >> 1) & 1] = add2(rs2[(i >> 1) & 1], pack_f2(e0, e1));
                         s[i >> 1] = pack_bf16x2(e0, e1);
                     }
                 };
-                if (p.causal && j == n_t - 1) exp_row(std::true_type{});
+                if (masked) exp_row(std::true_type{});
                 else exp_row(std::false_type{});
                 float ra, rb;
                 unpack_f2(add2(rs2[0], rs2[1]), ra, rb);
@@ -236,8 +243,8 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.l_full[t]);
             ++ep_cnt;
-            if (p.has_lse) {
-                const int s_pos = (2 * item.qb + t) * kTile + row;
+            const int s_pos = (2 * item.qb + t) * kTile + row;
+            if (p.has_lse && s_pos < p.S) {
                 p.lse[item.r][((size_t)item.bl * p.Hq_l + item.h) * p.S + s_pos] =
                     m_ref * 0.6931471805599453f + logf(l_run);
             }
@@ -287,6 +294,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 const TileCoord c = locate(p, item.r, item.bl, (2 * item.qb + t) * kTile, item.h, p.Hq_l);
                 __nv_bfloat16 *dst = p.o[c.rank] + ((size_t)(c.row + row) * p.o_heads + c.head) * D;
                 const uint32_t O_t = tmem + 256 + 128 * t + lane_addr;
+                const bool in_seq = (2 * item.qb + t) * kTile + row < p.S;   // rows past a ragged end are not stored
 #pragma unroll
                 for (int cc = 0; cc < kOCols / 32; ++cc) {
                     uint32_t rr[32];
@@ -299,7 +307,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                         o4.y = pack_bf16x2(__uint_as_float(rr[8 * i + 2]) * inv_l, __uint_as_float(rr[8 * i + 3]) * inv_l);
                         o4.z = pack_bf16x2(__uint_as_float(rr[8 * i + 4]) * inv_l, __uint_as_float(rr[8 * i + 5]) * inv_l);
                         o4.w = pack_bf16x2(__uint_as_float(rr[8 * i + 6]) * inv_l, __uint_as_float(rr[8 * i + 7]) * inv_l);
-                        *reinterpret_cast<uint4 *>(dst + cc * 32 + i * 8) = o4;
+                        if (in_seq) *reinterpret_cast<uint4 *>(dst + cc * 32 + i * 8) = o4;
                     }
                 }
                 tc_fence_before();

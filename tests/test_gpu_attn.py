@@ -43,6 +43,16 @@ def test_attn_fwd_matches_oracle(basp, name, w):
     assert np.abs(lse - ref_lse).max() < 2e-3, np.abs(lse - ref_lse).max()
 
 
+@pytest.mark.parametrize("S,causal", [(1, True), (77, True), (200, True), (333, False), (129, False), (1000, True)])
+def test_ragged_sequence_lengths(basp, S, causal):
+    """S not a multiple of the 128-row tile: the last tile is masked, rows past the end are not stored
+    (two sequences per rank, so what follows a ragged end is the next sequence, not padding)."""
+    w = synth.Workload("ragged_S", N=2, B=4, S=S, Hq=4, Hkv=2, D=128, G=2)
+    got, ref, lse, ref_lse = run_attn(basp, w, causal=causal, seed=S)
+    assert_attn_close(got, ref, f"S={S}")
+    assert np.abs(lse - ref_lse).max() < 2e-3
+
+
 def test_noncausal_and_explicit_scale(basp):
     w = synth.Workload("nc", N=2, B=2, S=384, Hq=4, Hkv=2, D=64)
     got, ref, lse, ref_lse = run_attn(basp, w, causal=False, scale=0.2, seed=5)

@@ -75,6 +75,8 @@ def test_null_and_alignment_checks_need_no_gpu(basp):
     assert L.basp_attn_fwd(pl.handle, good, good, good, good, None, 0.0, None) == basp.BASP_ERR_ALIAS
     assert L.basp_layer_fwd(pl.handle, good, good, good, good2, None, ctypes.c_void_p(0x1000), 16, 0.0, None) \
         == basp.BASP_ERR_WORKSPACE
-    pl2 = basp.basp_plan_create(4, 2, 1000, 8, 8, 64)    # S not a multiple of 128
-    assert L.basp_attn_fwd(pl2.handle, good, good, good, good2, None, 0.0, None) == basp.BASP_ERR_UNSUPPORTED
+    pl2 = basp.basp_plan_create(4, 2, 1000, 8, 8, 64)    # T = 500 is not a multiple of 128: tiles would straddle ranks
+    assert L.basp_layer_fwd_fused(pl2.handle, good, good, good, good2, None, 0.0, None) == basp.BASP_ERR_UNSUPPORTED
+    pl3 = basp.basp_plan_create(4, 2, 1024, 8, 8, 32)    # head dim the kernels do not implement
+    assert L.basp_attn_fwd(pl3.handle, good, good, good, good2, None, 0.0, None) == basp.BASP_ERR_UNSUPPORTED
     assert basp.lib.basp_strerror(-7).decode().startswith("a bounded wait")
