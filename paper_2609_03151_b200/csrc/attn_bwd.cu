@@ -151,6 +151,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         const int row = tid & 127;                      // TMEM lane: key row (scores) / query row (dQ)
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         uint32_t it_g = 0, item_n = 0;
+        int pending_stage = -1;                         // Q/dO stage whose dQ reduce-add is still in flight
         BwdItem item;
         for (int round = 0; bwd_get_item(p, round, item); ++round, ++item_n) {
             for (int hq = 0; hq < p.q_per_kv; ++hq) {
@@ -210,6 +211,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars->pds_ready);
+                    if (pending_stage >= 0 && lane == 0) {     // previous step's dQ block has left shared memory
+                        tma_store_wait_read<0>();
+                        mbar_arrive(&bars->qdo_empty[pending_stage]);
+                    }
 
                     // dQ_m tile: lane = query row, this quarter owns head-dim columns 32g .. 32g+31
                     BPH_T(t4);
@@ -242,10 +247,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                             tma_reduce_add_3d(&p.dq_acc[item.r], chunk + (warp & 3) * 4096, 32 * g, h,
                                               item.bl * p.S + m * kT + (warp & 3) * 32);
                             tma_store_commit();
-                            tma_store_wait_read<0>();
 #endif
-                            mbar_arrive(&bars->qdo_empty[stage]);
                         }
+                        // the stage is handed back one step later (after the next step's P^T / dS^T are out), when
+                        // the copy has long read it: the reduce-add runs under the next step's arithmetic
+                        pending_stage = (int)stage;
                     }
                     BPH_T(t6);
                     BPH_ADD(0, t0, t1); BPH_ADD(1, t1, t2); BPH_ADD(2, t2, t3); BPH_ADD(3, t3, t4);
@@ -280,6 +286,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->dkdv_read);
+        }
+        if (pending_stage >= 0 && lane == 0) {          // last step's reduce-add must have read shared memory
+            tma_store_wait_read<0>();
+            mbar_arrive(&bars->qdo_empty[pending_stage]);
         }
     } else if (warp == kBwdComputeWarps) {
         // ======================================================================= TMA producer
