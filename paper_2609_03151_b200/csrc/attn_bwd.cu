@@ -13,10 +13,12 @@
 //   (2) dP^T = V dO^T       SS   -> TMEM [128,256)
 //   compute warps: P^T = exp2(..), dS^T = scale P^T (dP^T - Delta)  ->  P^T bf16 to TMEM, dS^T bf16 to smem
 //   (3) dV  += P^T dO       TS   -> TMEM [384,512)
-//   (4) dK  += dS^T Q       SS   -> TMEM [256,384)
 //   (5) dQ_m = dS K         SS   -> TMEM [128,256)  (A = the dS^T buffer read MN-major)
-//   compute warps: dQ_m staged through the (now free) Q / dO stage and added to the fp32 accumulator in
-//   global memory by TMA reduce-add (order of the additions not fixed).
+//   (4) dK  += dS^T Q       SS   -> TMEM [256,384)
+//   drain warps: dQ_m staged through the (now free) Q / dO stage and added to the fp32 accumulator in
+//   global memory by TMA reduce-add (order of the additions not fixed), while the compute warps and
+//   the tensor core are already on the next step.
+// Warps: 16 compute (a quarter of the score columns each), 4 drain, TMA producer, MMA issuer.
 // Helper kernels: Delta = rowsum(dO * O); fp32 dQ accumulator -> bf16.
 #include <cuda.h>
 #include <math.h>
@@ -33,7 +35,10 @@ using namespace ptx;
 
 constexpr int kT = 128;
 constexpr int kBwdComputeWarps = 16;
-constexpr int kBwdThreads = (kBwdComputeWarps + 2) * 32;   // compute warps + TMA warp + MMA warp
+constexpr int kBwdDrainWarp0 = kBwdComputeWarps;          // 4 warps that take dQ out of TMEM and reduce-add it
+constexpr int kBwdTmaWarp = kBwdComputeWarps + 4;
+constexpr int kBwdMmaWarp = kBwdComputeWarps + 5;
+constexpr int kBwdThreads = (kBwdComputeWarps + 8) * 32;   // + drain warpgroup + (TMA, MMA, two idle warps)
 
 template <int R>
 struct BwdParams {
@@ -72,7 +77,7 @@ __device__ __forceinline__ bool bwd_get_item(const BwdParams<R> &p, int round, B
 
 struct BwdBars {
     uint64_t kv_full, kv_empty, qdo_full[2], qdo_empty[2], qdo_mma_done[2];
-    uint64_t s_full, stats_full, pds_ready, dq_full, dq_read, dkdv_full, dkdv_read;
+    uint64_t s_full, stats_full[2], pds_ready, dq_full, dq_read, dkdv_full, dkdv_read;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -88,7 +93,7 @@ __device__ __forceinline__ void bwd_report(int *status, int code, int role, int 
 #ifdef BASP_PHASE_TIMING
 __device__ long long g_bwd_phase[32];
 #define BPH_T(var) const long long var = clock64()
-#define BPH_ADD(slot, a, b) do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (warp == 0 || warp == kBwdComputeWarps + 1)) g_bwd_phase[slot] += (b) - (a); } while (0)
+#define BPH_ADD(slot, a, b) do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (warp == 0 || warp == kBwdMmaWarp || warp == kBwdDrainWarp0)) g_bwd_phase[slot] += (b) - (a); } while (0)
 #else
 #define BPH_T(var)
 #define BPH_ADD(slot, a, b)
@@ -123,21 +128,22 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         mbar_init(&bars->kv_full, 1); mbar_init(&bars->kv_empty, 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(&bars->qdo_full[s], 1);
-            mbar_init(&bars->qdo_empty[s], kBwdComputeWarps);   // every compute warp has drained its dQ block
+            mbar_init(&bars->qdo_empty[s], 4);                  // every drain warp's reduce-add has read the stage
             mbar_init(&bars->qdo_mma_done[s], 1);
         }
         mbar_init(&bars->s_full, 1);
-        mbar_init(&bars->stats_full, kBwdComputeWarps);
+        mbar_init(&bars->stats_full[0], 1);
+        mbar_init(&bars->stats_full[1], 1);
         mbar_init(&bars->pds_ready, kBwdComputeWarps);
         mbar_init(&bars->dq_full, 1);
-        mbar_init(&bars->dq_read, kBwdComputeWarps);
+        mbar_init(&bars->dq_read, 4);
         mbar_init(&bars->dkdv_full, 1);
         mbar_init(&bars->dkdv_read, kBwdComputeWarps);
         bars->abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         if (bars->abort_flag) bwd_report(p.status, 4, 0, (int)(smem_u32(smem) & 1023u));
         fence_mbar_init();
     }
-    if (warp == kBwdComputeWarps) { tmem_alloc(&bars->tmem_base, 512); tmem_relinquish(); }
+    if (warp == kBwdTmaWarp) { tmem_alloc(&bars->tmem_base, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -147,26 +153,20 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
 
     if (warp < kBwdComputeWarps) {
         // ======================================================================= compute warps
+        // (no register change: 16 warps x 80 registers; the pool that setmaxnreg redistributes is what the CTA got at
+        //  launch, 768 x 80, so 4 x 32 x 104 for the drain warps has to come out of the last warpgroup's 4 x 32 x 24)
         const int g = warp >> 2;                        // which 32-column quarter of the score tile
         const int row = tid & 127;                      // TMEM lane: key row (scores) / query row (dQ)
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         uint32_t it_g = 0, item_n = 0;
-        int pending_stage = -1;                         // Q/dO stage whose dQ reduce-add is still in flight
         BwdItem item;
         for (int round = 0; bwd_get_item(p, round, item); ++round, ++item_n) {
             for (int hq = 0; hq < p.q_per_kv; ++hq) {
                 const int h = item.hkv * p.q_per_kv + hq;
                 for (int m = item.m0; m < item.n_qt; ++m, ++it_g) {
                     const int buf = it_g & 1;
-                    {   // row statistics of the query tile: LSE (in log2 units) and Delta
-                        const size_t off = ((size_t)item.bl * p.Hq_l + h) * p.S + (size_t)m * kT + row;
-                        if (g == 0) s_lse[buf * kT + row] = p.lse[item.r][off] * 1.4426950408889634f;
-                        else if (g == 1) s_delta[buf * kT + row] = p.delta[item.r][off];
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&bars->stats_full);
-                    }
                     BPH_T(t0);
-                    BWD_WAIT(&bars->stats_full, it_g & 1, 10, m);
+                    BWD_WAIT(&bars->stats_full[buf], (it_g >> 1) & 1, 10, m);   // LSE and Delta of the query tile (producer warp)
                     BWD_WAIT(&bars->s_full, it_g & 1, 11, m);
                     tc_fence_after();
                     BPH_T(t1);
@@ -211,48 +211,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars->pds_ready);
-                    if (pending_stage >= 0 && lane == 0) {     // previous step's dQ block has left shared memory
-                        tma_store_wait_read<0>();
-                        mbar_arrive(&bars->qdo_empty[pending_stage]);
-                    }
-
-                    // dQ_m tile: lane = query row, this quarter owns head-dim columns 32g .. 32g+31
                     BPH_T(t4);
-                    BWD_WAIT(&bars->dq_full, it_g & 1, 12, m);
-                    tc_fence_after();
                     BPH_T(t5);
-                    uint32_t dq[32];
-                    tmem_ld_x32(tmem + kColDP + 32 * g + lane_addr, dq);
-                    tmem_wait_ld();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars->dq_read);
-                    // dQ leaves through the Q / dO stage of this step: once products (3) and (4) have read it, the
-                    // stage is 64 KiB of free shared memory = the fp32 dQ tile.  Quarter g owns the 16 KiB chunk g
-                    // ([128 rows][32 floats], 128-byte swizzle); each warp adds its own 32 rows with one TMA
-                    // reduce-add and releases the stage to the producer when the copy has read shared memory.
-                    {
-                        const uint32_t stage = it_g & 1, ph = (it_g >> 1) & 1;
-                        BWD_WAIT(&bars->qdo_mma_done[stage], ph, 14, m);
-                        uint8_t *chunk = (g < 2 ? sQ : sdO) + stage * kTileBytes + (g & 1) * 16384;
-                        uint8_t *line = chunk + row * 128;
-#pragma unroll
-                        for (int ch = 0; ch < 8; ++ch)
-                            *reinterpret_cast<uint4 *>(line + ((ch ^ (row & 7)) << 4)) =
-                                make_uint4(dq[4 * ch], dq[4 * ch + 1], dq[4 * ch + 2], dq[4 * ch + 3]);
-                        fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) {
-#ifndef BWD_NO_RED
-                            tma_reduce_add_3d(&p.dq_acc[item.r], chunk + (warp & 3) * 4096, 32 * g, h,
-                                              item.bl * p.S + m * kT + (warp & 3) * 32);
-                            tma_store_commit();
-#endif
-                        }
-                        // the stage is handed back one step later (after the next step's P^T / dS^T are out), when
-                        // the copy has long read it: the reduce-add runs under the next step's arithmetic
-                        pending_stage = (int)stage;
-                    }
                     BPH_T(t6);
                     BPH_ADD(0, t0, t1); BPH_ADD(1, t1, t2); BPH_ADD(2, t2, t3); BPH_ADD(3, t3, t4);
                     BPH_ADD(4, t4, t5); BPH_ADD(5, t5, t6); BPH_ADD(6, t0, t0 + 1);
@@ -287,11 +247,79 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->dkdv_read);
         }
-        if (pending_stage >= 0 && lane == 0) {          // last step's reduce-add must have read shared memory
-            tma_store_wait_read<0>();
-            mbar_arrive(&bars->qdo_empty[pending_stage]);
+    } else if (warp < kBwdTmaWarp) {
+        // ======================================================================= dQ drain warps
+        // dQ_m (lane = query row, 128 fp32 columns) leaves TMEM through the Q / dO stage of its step, which is
+        // 64 KiB of free shared memory once the products that read it are done: chunk c ([128 rows][32 floats],
+        // 128-byte swizzle) goes to the dO half (c = 2, 3; product (3) is complete when dQ is) or the Q half
+        // (c = 0, 1; after product (4)).  Each warp adds its 32 rows of a chunk with one TMA reduce-add.
+        reg_inc<104>();
+        const int wq = warp & 3;
+        const int row = tid & 127;
+        const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
+        uint32_t it_g = 0;
+        BwdItem item;
+        for (int round = 0; bwd_get_item(p, round, item); ++round) {
+            for (int hq = 0; hq < p.q_per_kv; ++hq) {
+                const int h = item.hkv * p.q_per_kv + hq;
+                for (int m = item.m0; m < item.n_qt; ++m, ++it_g) {
+                    const uint32_t stage = it_g & 1, ph = (it_g >> 1) & 1;
+                    BPH_T(v0);
+                    BWD_WAIT(&bars->dq_full, it_g & 1, 12, m);
+                    tc_fence_after();
+                    BPH_T(v1);
+                    uint32_t lo[64];
+                    auto stage_chunk = [&](int c, const uint32_t *v) {
+                        uint8_t *line = (c < 2 ? sQ : sdO) + stage * kTileBytes + (c & 1) * 16384 + row * 128;
+#pragma unroll
+                        for (int ch = 0; ch < 8; ++ch)
+                            *reinterpret_cast<uint4 *>(line + ((ch ^ (row & 7)) << 4)) =
+                                make_uint4(v[4 * ch], v[4 * ch + 1], v[4 * ch + 2], v[4 * ch + 3]);
+                    };
+                    {
+                        uint32_t hi[32];
+#pragma unroll
+                        for (int c = 2; c < 4; ++c) {
+                            tmem_ld_x32(tmem + kColDP + 32 * c + lane_addr, hi);
+                            tmem_wait_ld();
+                            stage_chunk(c, hi);
+                        }
+                    }
+                    tmem_ld_x32(tmem + kColDP + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&lo[0]));
+                    tmem_ld_x32(tmem + kColDP + 32 + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&lo[32]));
+                    tmem_wait_ld();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->dq_read);          // TMEM is free for the next dP^T
+                    BPH_T(v2);
+                    BWD_WAIT(&bars->qdo_mma_done[stage], ph, 14, m);     // product (4) has read the Q half
+                    BPH_T(v3);
+                    stage_chunk(0, &lo[0]);
+                    stage_chunk(1, &lo[32]);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+#ifndef BWD_NO_RED
+                    if (lane == 0) {
+                        const int row0 = item.bl * p.S + m * kT + wq * 32;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            tma_reduce_add_3d(&p.dq_acc[item.r],
+                                              (c < 2 ? sQ : sdO) + stage * kTileBytes + (c & 1) * 16384 + wq * 4096,
+                                              32 * c, h, row0);
+                        tma_store_commit();
+                        tma_store_wait_read<0>();          // these warps have nothing else to do until the next dQ tile
+                    }
+#endif
+                    if (lane == 0) mbar_arrive(&bars->qdo_empty[stage]);
+                    BPH_T(v4);
+                    BPH_ADD(16, v0, v1); BPH_ADD(17, v1, v2); BPH_ADD(18, v2, v3); BPH_ADD(19, v3, v4); BPH_ADD(20, v0, v0 + 1);
+                }
+            }
         }
-    } else if (warp == kBwdComputeWarps) {
+    } else {
+      // every warp of the last warpgroup gives registers back at this one place (TMA, MMA and two idle warps)
+      reg_dec<56>();
+      if (warp == kBwdTmaWarp) {
         // ======================================================================= TMA producer
         uint32_t it_g = 0, item_n = 0;
         BwdItem item;
@@ -318,10 +346,22 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                             tma_load_3d(sdO + stage * kTileBytes + s * 16384, &p.dout[item.r], &bars->qdo_full[stage], s * 64, h, row0);
                         }
                     }
+                    {   // row statistics of the query tile: LSE (to log2 units) and Delta, four rows per lane.  The buffer
+                        // has the stage's parity: its last readers (step it-2) finished before the stage was released.
+                        const size_t off = ((size_t)item.bl * p.Hq_l + h) * p.S + (size_t)m * kT + 4 * lane;
+                        float4 l4 = *reinterpret_cast<const float4 *>(p.lse[item.r] + off);
+                        const float4 d4 = *reinterpret_cast<const float4 *>(p.delta[item.r] + off);
+                        l4.x *= 1.4426950408889634f; l4.y *= 1.4426950408889634f;
+                        l4.z *= 1.4426950408889634f; l4.w *= 1.4426950408889634f;
+                        *reinterpret_cast<float4 *>(s_lse + stage * kT + 4 * lane) = l4;
+                        *reinterpret_cast<float4 *>(s_delta + stage * kT + 4 * lane) = d4;
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bars->stats_full[stage]);
+                    }
                 }
             }
         }
-    } else if (warp == kBwdComputeWarps + 1) {
+      } else if (warp == kBwdMmaWarp) {
         // ======================================================================= MMA issuer
         const uint32_t idesc_kk = make_idesc_bf16(kT, kT, false, false);     // (1) (2): both operands K-major
         const uint32_t idesc_kn = make_idesc_bf16(kT, D, false, true);       // (3) (4): B is MN-major
@@ -369,19 +409,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     tc_fence_after();
                     if (lane == 0) {
                         const uint32_t acc0 = first ? 0u : 1u;
-                        // (5) dQ_m = dS K : A = the dS^T buffer read MN-major (query rows), B = K MN-major.  Issued
-                        //     first so that the compute warps can take dQ out of TMEM while (3) and (4) run.
-#pragma unroll
-                        for (int kk = 0; kk < kT / 16; ++kk)
-                            mma_ss(tmem + kColDP, desc_mn | (uint64_t)(adS + kk * 128), desc_mn | (uint64_t)(aK + kk * 128),
-                                   idesc_nn, kk > 0);
-                        tc_commit(&bars->dq_full);
                         // (3) dV += P^T dO : A = P^T in TMEM (query index along K: 8 columns per 16 queries,
                         //     each quarter of 32 queries starts at its own column 32g), B = dO read MN-major
 #pragma unroll
                         for (int kk = 0; kk < kT / 16; ++kk)
                             mma_ts(tmem + kColDV, tmem + kColST + (kk / 2) * 32 + (kk % 2) * 8,
                                    desc_mn | (uint64_t)(do16 + kk * 128), idesc_kn, kk > 0 ? 1u : acc0);
+                        // (5) dQ_m = dS K : A = the dS^T buffer read MN-major (query rows), B = K MN-major.  When it is
+                        //     complete so is (3): the dO half of the stage is free for the drain warps.
+#pragma unroll
+                        for (int kk = 0; kk < kT / 16; ++kk)
+                            mma_ss(tmem + kColDP, desc_mn | (uint64_t)(adS + kk * 128), desc_mn | (uint64_t)(aK + kk * 128),
+                                   idesc_nn, kk > 0);
+                        tc_commit(&bars->dq_full);
                         // (4) dK += dS^T Q : A = dS^T from shared memory (K-major: query columns), B = Q MN-major
 #pragma unroll
                         for (int kk = 0; kk < kT / 16; ++kk) {
@@ -402,6 +442,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 tc_commit(&bars->kv_empty);
             }
         }
+      }
     }
 
 bwd_done:
@@ -412,7 +453,7 @@ bwd_done:
         while (globaltimer_ns() - t0 < 200000ull) { }
         __syncthreads();
     }
-    if (warp == kBwdComputeWarps) tmem_dealloc(tmem, 512);
+    if (warp == kBwdTmaWarp) tmem_dealloc(tmem, 512);
 }
 
 #undef BWD_WAIT
