@@ -236,6 +236,12 @@ size_t basp_host_arena_bytes(const basp_plan *plan);
 int basp_get_status(void *stream, int *status_out);
 int basp_clear_status(void *stream);
 
+/* Diagnostic: launches a one-CTA kernel whose wait cannot complete, with a wait limit of limit_us microseconds
+ * (1 .. 1 000 000), so that a caller can check that an expired wait is reported ({code 2, role 100, block, waited
+ * microseconds} through basp_get_status -> BASP_ERR_TIMEOUT) and that the context stays usable afterwards.  The
+ * kernel ends by itself; nothing faults.  Clear the status words afterwards with basp_clear_status. */
+int basp_selftest_wait_timeout(unsigned int limit_us, void *stream);
+
 const char *basp_strerror(int code);
 /* Text of the last CUDA error seen by the calling thread inside this library ("" if none). */
 const char *basp_last_cuda_error(void);

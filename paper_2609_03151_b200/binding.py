@@ -29,7 +29,7 @@ EXPORTS = [
     "basp_layer_fwd_host", "basp_host_arena_bytes", "basp_layer_fwd_static",
     "basp_layer_workspace_shards", "basp_attn_bwd", "basp_attn_bwd_workspace_bytes", "basp_reshard_grads_h2s",
     "basp_layer_bwd", "basp_layer_bwd_workspace_bytes", "basp_get_status", "basp_clear_status",
-    "basp_strerror", "basp_last_cuda_error", "basp_launch_count",
+    "basp_strerror", "basp_last_cuda_error", "basp_launch_count", "basp_selftest_wait_timeout",
 ]
 
 
@@ -76,6 +76,7 @@ lib.basp_host_arena_bytes.argtypes = [c_void_p]
 lib.basp_host_arena_bytes.restype = c_size_t
 lib.basp_get_status.argtypes = [c_void_p, POINTER(c_int)]
 lib.basp_clear_status.argtypes = [c_void_p]
+lib.basp_selftest_wait_timeout.argtypes = [ctypes.c_uint, c_void_p]
 lib.basp_strerror.argtypes = [c_int]
 lib.basp_strerror.restype = c_char_p
 lib.basp_last_cuda_error.restype = c_char_p
@@ -286,6 +287,10 @@ def basp_get_status(stream=None, raise_on_timeout=True):
 
 def basp_clear_status(stream=None):
     _check(lib.basp_clear_status(_stream(stream)), "basp_clear_status")
+
+
+def basp_selftest_wait_timeout(limit_us: int, stream=None):
+    _check(lib.basp_selftest_wait_timeout(int(limit_us), _stream(stream)), "basp_selftest_wait_timeout")
 
 
 def basp_launch_count() -> int:

@@ -35,7 +35,7 @@ using namespace ptx;
 
 constexpr int kT = 128;
 constexpr int kBwdComputeWarps = 16;
-constexpr int kBwdDrainWarp0 = kBwdComputeWarps;          // 4 warps that take dQ out of TMEM and reduce-add it
+[[maybe_unused]] constexpr int kBwdDrainWarp0 = kBwdComputeWarps;          // 4 warps that take dQ out of TMEM and reduce-add it
 constexpr int kBwdTmaWarp = kBwdComputeWarps + 4;
 constexpr int kBwdMmaWarp = kBwdComputeWarps + 5;
 constexpr int kBwdThreads = (kBwdComputeWarps + 8) * 32;   // + drain warpgroup + (TMA, MMA, two idle warps)

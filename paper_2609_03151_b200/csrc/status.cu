@@ -4,6 +4,7 @@
 #include <cstring>
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace {
 __device__ int g_basp_status[4];              // {code, role, block, detail}; 0 = fine
@@ -42,6 +43,44 @@ extern "C" int basp_clear_status(void *stream) {
     int *dev = basp_status_device_ptr();
     if (!dev) return BASP_ERR_CUDA;
     BASP_CUDA_TRY(cudaMemsetAsync(dev, 0, 4 * sizeof(int), (cudaStream_t)stream));
+    return BASP_OK;
+}
+
+namespace {
+// Two warps wait on a barrier that nothing ever arrives on: warp 0 with the given (short) limit, warp 1 with the
+// normal one.  Warp 0 gives up, records {code 2, role, block, detail = waited microseconds} and raises the CTA's abort
+// flag; warp 1 must then leave through that flag.  Both reach the final barrier: the kernel ends by itself.
+__global__ void wait_selftest_kernel(int *status, unsigned long long limit_ns) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    const uint64_t t0 = ptx::globaltimer_ns();
+    const bool ok = ptx::mbar_wait(&bar, 0, &abort_flag, 0, warp == 0 ? limit_ns : ptx::kWaitLimitNs);
+    if (!ok && warp == 0 && (threadIdx.x & 31) == 0) {
+        abort_flag = 1;
+        if (atomicCAS(status, 0, 2) == 0) {
+            status[1] = 100;
+            status[2] = (int)blockIdx.x;
+            status[3] = (int)((ptx::globaltimer_ns() - t0) / 1000);
+        }
+    }
+    __syncthreads();
+}
+}  // namespace
+
+extern "C" int basp_selftest_wait_timeout(unsigned int limit_us, void *stream) {
+    if (limit_us == 0 || limit_us > 1000000u) return BASP_ERR_INVALID;
+    int *dev = basp_status_device_ptr();
+    if (!dev) return BASP_ERR_CUDA;
+    wait_selftest_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(dev, (unsigned long long)limit_us * 1000ull);
+    BASP_CUDA_TRY(cudaGetLastError());
+    basp_count_launch(1);
     return BASP_OK;
 }
 
