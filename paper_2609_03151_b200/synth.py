@@ -62,6 +62,17 @@ WORKLOADS = {
 }
 
 
+# The paper's own sweep axes on one GPU (Section VI-C: S = 8K, micro-batch 1..8, Llama-3.2-1B, N = 8; Section VI-D:
+# S = 1K..32K, micro-batch 2, Llama-3.2-3B).  The paper's table gives hidden size and 32 heads only; the shapes below are
+# the public models' (1B: 32 query / 8 KV heads of 64; 3B: 24 / 8 heads of 128 -- 3072 / 32 = 96 is not a supported D).
+for _b in (1, 2, 4, 8):
+    WORKLOADS[f"e5_b{_b}_basp"] = Workload(f"e5_b{_b}_basp", N=8, B=_b, S=8192, Hq=32, Hkv=8, D=64)
+    WORKLOADS[f"e5_b{_b}_ulysses"] = Workload(f"e5_b{_b}_ulysses", N=8, B=_b, S=8192, Hq=32, Hkv=8, D=64, G=1)
+for _s in (1, 2, 4, 8, 16, 32):
+    WORKLOADS[f"e6_s{_s}k_basp"] = Workload(f"e6_s{_s}k_basp", N=8, B=2, S=_s * 1024, Hq=24, Hkv=8, D=128)
+    WORKLOADS[f"e6_s{_s}k_ulysses"] = Workload(f"e6_s{_s}k_ulysses", N=8, B=2, S=_s * 1024, Hq=24, Hkv=8, D=128, G=1)
+
+
 def shrink(w: Workload, T: int = 512, name: str | None = None) -> Workload:
     """Same rank/head structure with T tokens per rank (S = T*K)."""
     return Workload(name or f"{w.name}_T{T}", w.N, w.B, T * w.K, w.Hq, w.Hkv, w.D, w.G, w.train)
