@@ -245,13 +245,38 @@ def run_gpu(args, w: synth.Workload):
     ms_bwd = [statistics.mean(e[i].elapsed_time(e[i + 1]) for e in ev) for i in (3, 4, 5)] if train else None
     basp.basp_get_status()
 
+    proj = None
+    if args.proj:      # the projections on either side of the core (not part of the step): X W_qkv^T and O W_o^T
+        hidden = w.Hq * w.D
+        xs = [randn((Bl * T, hidden)) for _ in range(N)]
+        w_qkv = (torch.randn(((w.Hq + 2 * w.Hkv) * w.D, hidden), generator=gen, device=dev) / hidden ** 0.5).to(torch.bfloat16)
+        w_o = (torch.randn((hidden, w.Hq * w.D), generator=gen, device=dev) / hidden ** 0.5).to(torch.bfloat16)
+        ys = [torch.empty((Bl * T, hidden), dtype=torch.bfloat16, device=dev) for _ in range(N)]
+        pe = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        for it in range(args.warmup + args.steps):
+            if it == args.warmup:
+                pe[0].record()
+            basp.basp_qkv_proj(plan, hidden, xs, w_qkv, q_seq, k_seq, v_seq)
+        pe[1].record()
+        for it in range(args.steps):
+            basp.basp_out_proj(plan, hidden, o_seq, w_o, ys)
+        pe[2].record()
+        torch.cuda.synchronize()
+        basp.basp_get_status()
+        ms_qkv, ms_out = pe[0].elapsed_time(pe[1]) / args.steps, pe[1].elapsed_time(pe[2]) / args.steps
+        f_qkv = 2.0 * N * Bl * T * hidden * (w.Hq + 2 * w.Hkv) * w.D
+        f_out = 2.0 * N * Bl * T * hidden * w.Hq * w.D
+        proj = {"hidden": hidden, "qkv_ms": ms_qkv, "qkv_tflops": f_qkv / ms_qkv / 1e9, "out_ms": ms_out,
+                "out_tflops": f_out / ms_out / 1e9, "peak_sustained": peaks["bf16_sustained"]}
+        del xs, ys, w_qkv, w_o
+
     if args.quick:     # kernel timings only (what the ncu recipes in profiles/ run)
         clocks = sampler.stop() if sampler else None
         if rank == 0:
             print(json.dumps({"workload": w.name, "ms_per_step": total_ms / args.steps, "ms_s2h": ms_s2h,
                               "ms_attn": ms_attn, "ms_h2s": ms_h2s, "gpu_launches": launches,
                               "attn_tflops": w.attn_flops_fwd() / ms_attn / 1e9, "clocks": clocks,
-                              "bwd_ms_s2h_attn_h2s": ms_bwd,
+                              "bwd_ms_s2h_attn_h2s": ms_bwd, "projections": proj,
                               "attn_bwd_tflops": (w.attn_flops_bwd() / ms_bwd[1] / 1e9) if train else None}), flush=True)
         pdist.finalize()
         return
@@ -395,6 +420,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="basp", choices=["basp", "reference"])
+    ap.add_argument("--proj", action="store_true", help="also time the QKV and output projection GEMMs (with --quick)")
     ap.add_argument("--quick", action="store_true", help="time the three kernels only (for profiler runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)

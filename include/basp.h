@@ -228,6 +228,21 @@ int basp_layer_fwd_host(const basp_plan *plan, const void *const *q_seq_host,
                         float softmax_scale, void *stream);
 size_t basp_host_arena_bytes(const basp_plan *plan);
 
+/* ---- the projections on either side of the attention core (Section II-A: Q = X W_Q, K = X W_K, V = X W_V for
+ * every head, MultiHead = Concat(H_1..H_h) W_O), applied to every rank's sequence shard in one launch.
+ *   basp_qkv_proj:  [Q | K | V]_r = X_r . W_qkv^T   X_r: bf16 [Bl*T][hidden] (rank r's tokens), W_qkv: bf16
+ *                   [(Hq + 2 Hkv) * D][hidden] (rows: W_Q's heads, then W_K's, then W_V's); the three column blocks
+ *                   are written to q_seq[r] ([Bl][T][Hq][D]), k_seq[r], v_seq[r] ([Bl][T][Hkv][D]): the layout
+ *                   basp_reshard_qkv_s2h and basp_layer_fwd_fused read.
+ *   basp_out_proj:  Y_r = O_r . W_o^T               O_r: bf16 [Bl*T][Hq*D] (the layer's sequence-sharded output),
+ *                   W_o: bf16 [hidden][Hq*D], Y_r: bf16 [Bl*T][hidden].
+ * bf16 operands, fp32 accumulation, bf16 results.  Requires hidden a multiple of 64 (qkv) / 256 (out) and
+ * Hq*D, Hkv*D multiples of 256, else BASP_ERR_UNSUPPORTED.  Weights are shared by all ranks (one device pointer). */
+int basp_qkv_proj(const basp_plan *plan, int hidden, const void *const *x_seq, const void *w_qkv,
+                  void *const *q_seq, void *const *k_seq, void *const *v_seq, void *stream);
+int basp_out_proj(const basp_plan *plan, int hidden, const void *const *o_seq, const void *w_o,
+                  void *const *y_seq, void *stream);
+
 /* ---- device status.  Every wait inside the kernels (on a shared-memory barrier) is bounded;
  * when one expires the kernel records where, lets its copies drain, frees its tensor memory
  * and returns.  basp_get_status synchronises `stream`, copies the four status words of the

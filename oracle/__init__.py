@@ -258,6 +258,13 @@ def layer_fwd(Xq: np.ndarray, Xk: np.ndarray, Xv: np.ndarray, pl: Plan,
                 o_head=oh, lse_head=lse, o_seq=os_, o_global=gather(os_, pl))
 
 
+# ------------------------------------------------------------------- projections
+def linear(X: np.ndarray, W: np.ndarray) -> np.ndarray:
+    """The projections of Section II-A (Q = X W_Q, ..., Concat(H_i) W_O) as one product in fp64:
+    X [M,K] and W [N,K] are bf16 bit patterns (W holds one output feature per row); returns X . W^T [M,N]."""
+    return bf16_bits_to_f64(X) @ bf16_bits_to_f64(W).T
+
+
 # ----------------------------------------------------------------- bf16 helpers
 def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
     """Exact widening of bf16 bit patterns to fp64."""

@@ -29,7 +29,7 @@ EXPORTS = [
     "basp_layer_fwd_host", "basp_host_arena_bytes", "basp_layer_fwd_static",
     "basp_layer_workspace_shards", "basp_attn_bwd", "basp_attn_bwd_workspace_bytes", "basp_reshard_grads_h2s",
     "basp_layer_bwd", "basp_layer_bwd_workspace_bytes", "basp_get_status", "basp_clear_status",
-    "basp_strerror", "basp_last_cuda_error", "basp_launch_count", "basp_selftest_wait_timeout",
+    "basp_strerror", "basp_last_cuda_error", "basp_launch_count", "basp_selftest_wait_timeout", "basp_qkv_proj", "basp_out_proj",
 ]
 
 
@@ -77,6 +77,8 @@ lib.basp_host_arena_bytes.restype = c_size_t
 lib.basp_get_status.argtypes = [c_void_p, POINTER(c_int)]
 lib.basp_clear_status.argtypes = [c_void_p]
 lib.basp_selftest_wait_timeout.argtypes = [ctypes.c_uint, c_void_p]
+lib.basp_qkv_proj.argtypes = [c_void_p, c_int, _PP, c_void_p, _PP, _PP, _PP, c_void_p]
+lib.basp_out_proj.argtypes = [c_void_p, c_int, _PP, c_void_p, _PP, c_void_p]
 lib.basp_strerror.argtypes = [c_int]
 lib.basp_strerror.restype = c_char_p
 lib.basp_last_cuda_error.restype = c_char_p
@@ -287,6 +289,18 @@ def basp_get_status(stream=None, raise_on_timeout=True):
 
 def basp_clear_status(stream=None):
     _check(lib.basp_clear_status(_stream(stream)), "basp_clear_status")
+
+
+def basp_qkv_proj(plan, hidden, x_seq, w_qkv, q_seq, k_seq, v_seq, stream=None):
+    n = plan.N
+    _check(lib.basp_qkv_proj(plan.handle, int(hidden), _ptrs(x_seq, n), c_void_p(w_qkv.data_ptr()), _ptrs(q_seq, n),
+                             _ptrs(k_seq, n), _ptrs(v_seq, n), _stream(stream)), "basp_qkv_proj")
+
+
+def basp_out_proj(plan, hidden, o_seq, w_o, y_seq, stream=None):
+    n = plan.N
+    _check(lib.basp_out_proj(plan.handle, int(hidden), _ptrs(o_seq, n), c_void_p(w_o.data_ptr()), _ptrs(y_seq, n),
+                             _stream(stream)), "basp_out_proj")
 
 
 def basp_selftest_wait_timeout(limit_us: int, stream=None):

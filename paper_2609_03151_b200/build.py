@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libbasp.so")
-SOURCES = ["plan.cpp", "status.cu", "reshard.cu", "attn_fwd.cu", "attn_bwd.cu", "layer.cu", "layer_static.cu"]
+SOURCES = ["plan.cpp", "status.cu", "reshard.cu", "attn_fwd.cu", "attn_bwd.cu", "proj_gemm.cu", "layer.cu", "layer_static.cu"]
 
 
 def _nvcc() -> str:
