@@ -72,8 +72,10 @@ __device__ __forceinline__ bool ws_get_item(const AttnParams<R> &p, int round, W
 struct WsShared {
     uint64_t q_full, q_empty;
     uint64_t kv_full[kStages], kv_empty[kStages];
-    uint64_t s_full[2], alpha_full[2], p_full[2], o_rescaled[2], o_final[2], l_full[2], o_free[2];
-    float alpha[2][kTile];
+    uint64_t s_free, pv_done[2];
+    uint64_t alpha_full[2][2];       // [tile][step parity]
+    uint64_t s_full[2], p_full[2], o_rescaled[2], o_final[2], l_full[2], o_free[2];
+    float alpha[2][2][kTile];        // [tile][step parity][row]
     float l[2][kTile];
     uint32_t tmem_base;
     int abort_flag;
@@ -83,11 +85,15 @@ struct WsShared {
 __device__ long long g_phase_cycles[64];
 #define PHASE_T(var) const long long var = clock64()
 #define PHASE_ADD(slot, a, b) do { if (blockIdx.x == 0 && (threadIdx.x & 127) == 0) g_phase_cycles[slot] += (b) - (a); } while (0)
-#define PHASE_ADD1(slot, a, b) do { if (blockIdx.x == 0) g_phase_cycles[slot] += (b) - (a); } while (0)
+#define PHASE_ADD1(slot, a, b) do { ph_acc[(slot) - 16] += (b) - (a); } while (0)
+#define PHASE_DECL long long ph_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}
+#define PHASE_FLUSH do { if (blockIdx.x == 0 && lane == 0) for (int i_ = 0; i_ < 8; ++i_) g_phase_cycles[16 + i_] = ph_acc[i_]; } while (0)
 #else
 #define PHASE_T(var)
 #define PHASE_ADD(slot, a, b)
 #define PHASE_ADD1(slot, a, b)
+#define PHASE_DECL
+#define PHASE_FLUSH
 #endif
 
 #ifndef BASP_SLEEP_NS
@@ -123,13 +129,17 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
         for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], 1); }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&sh.s_full[t], 1);
-            mbar_init(&sh.alpha_full[t], 4);
+            mbar_init(&sh.alpha_full[t][0], 4);
+            mbar_init(&sh.alpha_full[t][1], 4);
             mbar_init(&sh.p_full[t], 4);
             mbar_init(&sh.o_rescaled[t], 4);
             mbar_init(&sh.o_final[t], 1);
             mbar_init(&sh.l_full[t], 4);
             mbar_init(&sh.o_free[t], 4);
         }
+        mbar_init(&sh.s_free, 4);
+        mbar_init(&sh.pv_done[0], 1);
+        mbar_init(&sh.pv_done[1], 1);
         sh.abort_flag = 0;
         fence_mbar_init();
     }
@@ -138,7 +148,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sh.tmem_base;
-    // S_t at columns 128 t, O_t at 256 + 128 t (only kOCols of them used); P_t overlays S_t.
+    // One score tile S at columns 0..127 (the two query tiles take turns), P_t at 128 + 64 t, O_t at 256 + 128 t.
 
     if (warp < 8) {
         // =============================================================== softmax of query tile t
@@ -146,7 +156,8 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
         const int t = warp >> 2;
         const int row = tid & 127;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t S_t = tmem + 128 * t + lane_addr;
+        const uint32_t S_a = tmem + lane_addr;                   // the shared score tile
+        const uint32_t P_t = tmem + 128 + 64 * t + lane_addr;
         uint32_t it_cnt = 0, ep_cnt = 0;
         WsItem item;
         for (int round = 0; ws_get_item(p, round, item); ++round) {
@@ -159,11 +170,14 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 tc_fence_after();
                 PHASE_T(c1);
                 uint32_t s[kTile];
-                tmem_ld_x32(S_t + 0, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-                tmem_ld_x32(S_t + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
-                tmem_ld_x32(S_t + 64, *reinterpret_cast<uint32_t(*)[32]>(&s[64]));
-                tmem_ld_x32(S_t + 96, *reinterpret_cast<uint32_t(*)[32]>(&s[96]));
+                tmem_ld_x32(S_a + 0, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+                tmem_ld_x32(S_a + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+                tmem_ld_x32(S_a + 64, *reinterpret_cast<uint32_t(*)[32]>(&s[64]));
+                tmem_ld_x32(S_a + 96, *reinterpret_cast<uint32_t(*)[32]>(&s[96]));
                 tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.s_free);       // the scores are in registers: the other tile's Q.K^T may overwrite S
                 PHASE_T(c2);
                 // Key column i of this tile is visible iff i <= lim: the causal diagonal (i <= row) and, in a
                 // ragged last tile, the end of the sequence (i < S - 128 j; what lies beyond belongs to the next
@@ -194,9 +208,9 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 if (j == 0) { m_new = mx; alpha = 1.f; }
                 else if (mx > m_ref + kRescaleThreshold) { m_new = mx; alpha = exp2_approx(m_ref - m_new); }
                 else { m_new = m_ref; alpha = 1.f; }
-                sh.alpha[t][row] = alpha;
+                sh.alpha[t][it_cnt & 1][row] = alpha;
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.alpha_full[t]);
+                if (lane == 0) mbar_arrive(&sh.alpha_full[t][it_cnt & 1]);
                 m_ref = m_new;
                 PHASE_T(c3);
                 const uint64_t sc2 = pack_f2(p.scale_log2, p.scale_log2), nm2 = pack_f2(-m_new, -m_new);
@@ -229,8 +243,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 unpack_f2(add2(rs2[0], rs2[1]), ra, rb);
                 l_run = l_run * alpha + (ra + rb);
                 PHASE_T(c4);
-                tmem_st_x32(S_t + 0, *reinterpret_cast<const uint32_t(*)[32]>(&s[0]));
-                tmem_st_x32(S_t + 32, *reinterpret_cast<const uint32_t(*)[32]>(&s[32]));
+                // P_t V(j-1) is issued behind Q_t K(j): make sure it has read P_t before P_t(j) replaces it
+                if (j > 0) { WS_WAIT(&sh.pv_done[t], (it_cnt - 1) & 1, 14 + t, j); tc_fence_after(); }
+                tmem_st_x32(P_t + 0, *reinterpret_cast<const uint32_t(*)[32]>(&s[0]));
+                tmem_st_x32(P_t + 32, *reinterpret_cast<const uint32_t(*)[32]>(&s[32]));
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
@@ -261,9 +277,13 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     if (j >= item.n[t]) continue;
-                    WS_WAIT(&sh.alpha_full[t], it_cnt[t] & 1, 20 + t, j);
+                    // two barriers per tile, used in turn: the softmax warps can be a step ahead of this one
+                    WS_WAIT(&sh.alpha_full[t][it_cnt[t] & 1], (it_cnt[t] >> 1) & 1, 20 + t, j);
+                    const float alpha = sh.alpha[t][it_cnt[t] & 1][row];
                     ++it_cnt[t];
-                    const float alpha = sh.alpha[t][row];
+                    // O_t is only ours once P_t V(j-1) has completed (it is issued behind Q_t K(j)); waiting for it
+                    // every step also keeps o_rescaled at most one phase ahead of the MMA warp
+                    if (j > 0) WS_WAIT(&sh.pv_done[t], (it_cnt[t] - 2) & 1, 22 + t, j);
                     if (j > 0 && !__all_sync(0xffffffffu, alpha == 1.f)) {
                         tc_fence_after();
                         const uint32_t O_t = tmem + 256 + 128 * t + lane_addr;
@@ -347,91 +367,88 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 }
             }
         } else if (warp == 13) {
-            // =========================================================== MMA issuer (lane 0 issues)
+            // =========================================================== MMA issuer 1: S = Q_t K_j^T (lane 0 issues)
+            // The two issuers run on their own barriers, so the tensor pipe takes whichever product is ready:
+            // Q_t.K(j+1) goes ahead as soon as the previous scores have been read out of the single S buffer,
+            // while P_t.V(j) waits for the softmax of step j.
             const uint32_t idesc_qk = make_idesc_bf16(kTile, kTile, false, false);
-            const uint32_t idesc_pv = make_idesc_bf16(kTile, D, false, true);
-            uint32_t kv_it = 0, item_n = 0, it_cnt[2] = {0, 0}, ep_cnt[2] = {0, 0};
-                WsItem item;
+            uint32_t item_n = 0, qk_cnt = 0, kv_base = 0;     // K_j of the item at ring index kv_base + 2j
+            WsItem item;
             // Descriptors differ only in the 14-bit start-address field, so a step along K is an add.
             const uint64_t desc_k = make_smem_desc_sw128(0, 16, 1024);        // K-major operands (Q, K)
-            const uint64_t desc_v = make_smem_desc_sw128(0, 16384, 1024);     // MN-major operand (V)
             const uint32_t q_addr16 = smem_u32(sQ) >> 4, kv_addr16 = smem_u32(sKV) >> 4;
-            auto issue_qk = [&](int t, uint32_t slot) {
-                const uint64_t a = desc_k | (uint64_t)(q_addr16 + t * (kTileBytes >> 4));
-                const uint64_t b = desc_k | (uint64_t)(kv_addr16 + slot * (kTileBytes >> 4));
-                if (lane == 0) {
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t off16 = ((kk / 4) * 16384 + (kk % 4) * 32) >> 4;
-                        mma_ss(tmem + 128 * t, a + off16, b + off16, idesc_qk, kk > 0);
-                    }
-                    tc_commit(&sh.s_full[t]);
-                }
-            };
-            auto commit = [&](uint64_t *bar) { if (lane == 0) tc_commit(bar); };
+            PHASE_DECL;
             for (int round = 0; ws_get_item(p, round, item); ++round, ++item_n) {
                 WS_WAIT(&sh.q_full, item_n & 1, 40, round);
-                uint32_t slot_k = kv_it % kStages;
-                WS_WAIT(&sh.kv_full[slot_k], (kv_it / kStages) & 1, 41, 0);
-                ++kv_it;
-                tc_fence_after();
-                for (int t = 0; t < 2; ++t)
-                    if (item.n[t] > 0) issue_qk(t, slot_k);
-                commit(&sh.kv_empty[slot_k]);
-                if (item.n_max == 1) commit(&sh.q_empty);
                 for (int j = 0; j < item.n_max; ++j) {
-                    const uint32_t slot_v = kv_it % kStages;
-                    PHASE_T(e0);
-                    WS_WAIT(&sh.kv_full[slot_v], (kv_it / kStages) & 1, 42, j);
-                    PHASE_T(e1);
-                    PHASE_ADD1(21, e0, e1); PHASE_ADD1(23, e0, e0 + 1);
-                    ++kv_it;
-                    const bool has_next = j + 1 < item.n_max;
-                    bool next_ready = false;
-                    if (has_next) { slot_k = kv_it % kStages; }
-                    const int last_v = j < item.n[1] ? 1 : 0;               // last tile that reads V_j
-                    const int last_k = (j + 1) < item.n[1] ? 1 : 0;         // last tile that reads K_{j+1}
-                    for (int t = 0; t < 2; ++t) {
-                        if (j < item.n[t]) {
-                            PHASE_T(d0);
-                            if (j == 0) WS_WAIT(&sh.o_free[t], (ep_cnt[t] & 1) ^ 1, 43 + t, round);
-                            PHASE_T(d1);
-                            WS_WAIT(&sh.p_full[t], it_cnt[t] & 1, 45 + t, j);
-                            PHASE_T(d2);
-                            WS_WAIT(&sh.o_rescaled[t], it_cnt[t] & 1, 47 + t, j);
-                            PHASE_T(d3);
-                            ++it_cnt[t];
-                            tc_fence_after();
-                            const uint64_t b = desc_v | (uint64_t)(kv_addr16 + slot_v * (kTileBytes >> 4));
-                            if (lane == 0) {
+                    const uint32_t idx = kv_base + 2 * j, slot = idx % kStages;
+                    PHASE_T(k0);
+                    WS_WAIT(&sh.kv_full[slot], (idx / kStages) & 1, 41, j);
+                    PHASE_T(k1);
+                    PHASE_ADD1(21, k0, k1);
+                    tc_fence_after();
 #pragma unroll
-                                for (int kk = 0; kk < kTile / 16; ++kk)
-                                    mma_ts(tmem + 256 + 128 * t, tmem + 128 * t + kk * 8, b + kk * (2048 >> 4), idesc_pv,
-                                           (j > 0) || (kk > 0));
+                    for (int t = 0; t < 2; ++t) {
+                        if (j >= item.n[t]) continue;
+                        // score tile number q may only follow the hand-over of q - 1 to its softmax warps
+                        PHASE_T(q0);
+                        if (qk_cnt > 0) { WS_WAIT(&sh.s_free, (qk_cnt - 1) & 1, 48, j); tc_fence_after(); }
+                        PHASE_T(q1);
+                        ++qk_cnt;
+                        const uint64_t a = desc_k | (uint64_t)(q_addr16 + t * (kTileBytes >> 4));
+                        const uint64_t b = desc_k | (uint64_t)(kv_addr16 + slot * (kTileBytes >> 4));
+                        if (lane == 0) {
+#pragma unroll
+                            for (int kk = 0; kk < D / 16; ++kk) {
+                                const uint32_t off16 = ((kk / 4) * 16384 + (kk % 4) * 32) >> 4;
+                                mma_ss(tmem, a + off16, b + off16, idesc_qk, kk > 0);
                             }
-                            if (j == item.n[t] - 1) { commit(&sh.o_final[t]); ++ep_cnt[t]; }
-                            PHASE_T(d4);
-                            PHASE_ADD1(16, d0, d1); PHASE_ADD1(17 + t, d1, d2); PHASE_ADD1(19, d2, d3); PHASE_ADD1(20, d3, d4);
+                            tc_commit(&sh.s_full[t]);
                         }
-                        if (t == last_v) commit(&sh.kv_empty[slot_v]);
-                        if (j + 1 < item.n[t]) {
-                            if (!next_ready) {
-                                PHASE_T(f0);
-                                WS_WAIT(&sh.kv_full[slot_k], (kv_it / kStages) & 1, 49, j);
-                                PHASE_T(f1);
-                                PHASE_ADD1(22, f0, f1);
-                                ++kv_it;
-                                next_ready = true;
-                                tc_fence_after();
-                            }
-                            issue_qk(t, slot_k);
-                            if (t == last_k) {
-                                commit(&sh.kv_empty[slot_k]);
-                                if (j + 2 == item.n_max) commit(&sh.q_empty);   // that was the item's last Q.K^T
-                            }
-                        }
+                        PHASE_T(q2);
+                        PHASE_ADD1(16, q0, q1); PHASE_ADD1(22, q1, q2); PHASE_ADD1(23, q0, q0 + 1);
+                    }
+                    if (lane == 0) {
+                        tc_commit(&sh.kv_empty[slot]);                            // K_j has no reader left
+                        if (j == item.n_max - 1) tc_commit(&sh.q_empty);          // that was the item's last Q.K^T
                     }
                 }
+                kv_base += 2 * item.n_max;
+            }
+            PHASE_FLUSH;
+        } else if (warp == 14) {
+            // =========================================================== MMA issuer 2: O_t += P_t V_j (lane 0 issues)
+            const uint32_t idesc_pv = make_idesc_bf16(kTile, D, false, true);
+            uint32_t it_cnt[2] = {0, 0}, ep_cnt[2] = {0, 0}, kv_base = 0;     // V_j at ring index kv_base + 2j + 1
+            WsItem item;
+            const uint64_t desc_v = make_smem_desc_sw128(0, 16384, 1024);     // MN-major operand (V)
+            const uint32_t kv_addr16 = smem_u32(sKV) >> 4;
+            for (int round = 0; ws_get_item(p, round, item); ++round) {
+                for (int j = 0; j < item.n_max; ++j) {
+                    const uint32_t idx = kv_base + 2 * j + 1, slot = idx % kStages;
+                    WS_WAIT(&sh.kv_full[slot], (idx / kStages) & 1, 42, j);
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        if (j >= item.n[t]) continue;
+                        if (j == 0) WS_WAIT(&sh.o_free[t], (ep_cnt[t] & 1) ^ 1, 43 + t, round);
+                        WS_WAIT(&sh.p_full[t], it_cnt[t] & 1, 45 + t, j);
+                        WS_WAIT(&sh.o_rescaled[t], it_cnt[t] & 1, 47 + t, j);
+                        ++it_cnt[t];
+                        tc_fence_after();
+                        const uint64_t b = desc_v | (uint64_t)(kv_addr16 + slot * (kTileBytes >> 4));
+                        if (lane == 0) {
+#pragma unroll
+                            for (int kk = 0; kk < kTile / 16; ++kk)
+                                mma_ts(tmem + 256 + 128 * t, tmem + 128 + 64 * t + kk * 8, b + kk * (2048 >> 4), idesc_pv,
+                                       (j > 0) || (kk > 0));
+                            tc_commit(&sh.pv_done[t]);
+                            if (j == item.n[t] - 1) tc_commit(&sh.o_final[t]);
+                        }
+                        if (j == item.n[t] - 1) ++ep_cnt[t];
+                    }
+                    if (lane == 0) tc_commit(&sh.kv_empty[slot]);                 // V_j has no reader left
+                }
+                kv_base += 2 * item.n_max;
             }
         }
     }
