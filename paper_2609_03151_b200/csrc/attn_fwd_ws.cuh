@@ -7,10 +7,16 @@
 //   warps  8-11  correction: rescales the O accumulators in TMEM when a row's reference maximum
 //                moved, and writes the normalised O tile at the end of the item
 //   warp  12     TMA producer (Q tiles, then K_0 V_0 K_1 V_1 ... through a shared-memory ring)
-//   warp  13     tcgen05.mma issuer (one thread)
-// While the softmax warps of one tile work on S_t(j), the tensor core runs P.V and the next
-// Q.K^T of the other tile.  TMEM: S_0 | S_1 | O_0 | O_1 (P_t as bf16 over the first 64 columns of
-// S_t).  All hand-offs are mbarriers; every wait is bounded.
+//   warp  13     tcgen05.mma issuer for S = Q_t K_j^T (one thread)
+//   warp  14     tcgen05.mma issuer for O_t += P_t V_j (one thread)
+// TMEM: S | P_0 P_1 | O_0 | O_1.  There is ONE score buffer: a softmax warp moves its row of S into
+// registers and hands the buffer back at once, so the next product (the other tile's, then this
+// tile's next key block) is computed while the exponentials run; P_t has columns of its own.  The two
+// issuers only follow their own barriers (scores read out / K tile landed; P_t written / O_t
+// rescaled / V tile landed), so the tensor pipe takes whichever product is ready and neither issuer's
+// waits sit in front of the other's work.  With one issuer and S_t overlaid by P_t the chain
+// softmax(j) -> P.V(j) -> Q.K(j+1) -> softmax(j+1) of a tile was serial and set the period.
+// All hand-offs are mbarriers; every wait is bounded.
 //
 // Online softmax with a lazily updated reference: the running reference m of a row only moves
 // when the tile maximum exceeds it by more than 8 (log2 units), so most iterations need no
@@ -29,7 +35,7 @@ constexpr float kRescaleThreshold = 8.f;
 #ifndef BASP_POLY_PAIRS
 #define BASP_POLY_PAIRS 0
 #endif
-constexpr int kPolyPairsOf4 = BASP_POLY_PAIRS;   // of every 4 score pairs, how many take the polynomial exp2
+constexpr int kPolyPairsOf8 = BASP_POLY_PAIRS;   // of every 8 score pairs, how many take the polynomial exp2
 
 struct WsItem {
     int r, bl, h, hkv, qb;
@@ -221,7 +227,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                     for (int i = 0; i < kTile; i += 2) {
                         const uint64_t x2 = fma2(pack_f2(__uint_as_float(s[i]), __uint_as_float(s[i + 1])), sc2, nm2);
                         float e0, e1;
-                        if (((i >> 1) & 3) < kPolyPairsOf4) {
+                        if (((i >> 1) & 7) < kPolyPairsOf8) {
                             exp2_poly_pair(x2, e0, e1);
                         } else {
                             float x0, x1;
