@@ -80,9 +80,10 @@ struct WsShared {
     uint64_t kv_full[kStages], kv_empty[kStages];
     uint64_t s_free, pv_done[2];
     uint64_t alpha_full[2][2];       // [tile][step parity]
-    uint64_t s_full[2], p_full[2], o_rescaled[2], o_final[2], l_full[2], o_free[2];
+    uint64_t s_full[2], p_full[2], o_rescaled[2], o_final[2], o_free[2];
+    uint64_t l_full[2][2];           // [tile][item parity]: a one-step item can end before the epilogue of the one before
     float alpha[2][2][kTile];        // [tile][step parity][row]
-    float l[2][kTile];
+    float l[2][2][kTile];            // [item parity][tile][row]
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -140,7 +141,8 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
             mbar_init(&sh.p_full[t], 4);
             mbar_init(&sh.o_rescaled[t], 4);
             mbar_init(&sh.o_final[t], 1);
-            mbar_init(&sh.l_full[t], 4);
+            mbar_init(&sh.l_full[t][0], 4);
+            mbar_init(&sh.l_full[t][1], 4);
             mbar_init(&sh.o_free[t], 4);
         }
         mbar_init(&sh.s_free, 4);
@@ -249,8 +251,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 unpack_f2(add2(rs2[0], rs2[1]), ra, rb);
                 l_run = l_run * alpha + (ra + rb);
                 PHASE_T(c4);
-                // P_t V(j-1) is issued behind Q_t K(j): make sure it has read P_t before P_t(j) replaces it
-                if (j > 0) { WS_WAIT(&sh.pv_done[t], (it_cnt - 1) & 1, 14 + t, j); tc_fence_after(); }
+                // The previous P_t V (of this item or, at j = 0, the last one of the item before) is issued by a warp
+                // of its own: make sure it has read P_t before this step's P_t replaces it.  Waiting at every step
+                // also means that no phase of the barrier is ever skipped.
+                if (it_cnt > 0) { WS_WAIT(&sh.pv_done[t], (it_cnt - 1) & 1, 14 + t, j); tc_fence_after(); }
                 tmem_st_x32(P_t + 0, *reinterpret_cast<const uint32_t(*)[32]>(&s[0]));
                 tmem_st_x32(P_t + 32, *reinterpret_cast<const uint32_t(*)[32]>(&s[32]));
                 tmem_wait_st();
@@ -261,9 +265,9 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 PHASE_ADD(8 * t + 0, c0, c1); PHASE_ADD(8 * t + 1, c1, c2); PHASE_ADD(8 * t + 2, c2, c3);
                 PHASE_ADD(8 * t + 3, c3, c4); PHASE_ADD(8 * t + 4, c4, c5); PHASE_ADD(8 * t + 5, c0, c0 + 1);
             }
-            sh.l[t][row] = l_run;
+            sh.l[ep_cnt & 1][t][row] = l_run;
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.l_full[t]);
+            if (lane == 0) mbar_arrive(&sh.l_full[t][ep_cnt & 1]);
             ++ep_cnt;
             const int s_pos = (2 * item.qb + t) * kTile + row;
             if (p.has_lse && s_pos < p.S) {
@@ -312,11 +316,11 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
                 if (item.n[t] == 0) continue;
-                WS_WAIT(&sh.l_full[t], ep_cnt[t] & 1, 24 + t, 0);
+                WS_WAIT(&sh.l_full[t][ep_cnt[t] & 1], (ep_cnt[t] >> 1) & 1, 24 + t, 0);
                 WS_WAIT(&sh.o_final[t], ep_cnt[t] & 1, 26 + t, 0);
+                const float inv_l = 1.f / sh.l[ep_cnt[t] & 1][t][row];
                 ++ep_cnt[t];
                 tc_fence_after();
-                const float inv_l = 1.f / sh.l[t][row];
                 const TileCoord c = locate(p, item.r, item.bl, (2 * item.qb + t) * kTile, item.h, p.Hq_l);
                 __nv_bfloat16 *dst = p.o[c.rank] + ((size_t)(c.row + row) * p.o_heads + c.head) * D;
                 const uint32_t O_t = tmem + 256 + 128 * t + lane_addr;
