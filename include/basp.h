@@ -173,6 +173,34 @@ int basp_layer_fwd_fused(const basp_plan *plan, const void *const *q_seq, const 
                          const void *const *v_seq, void *const *o_seq, float *const *lse_shards,
                          float softmax_scale, void *stream);
 
+/* ---- one physical GPU's share of the path when the n_ranks ranks are spread over several GPUs (Section IV-A:
+ * contiguous ranks per GPU; Section IV-C: the exchanges stay inside a group).  Every call takes the same host arrays
+ * of n_ranks device pointers as its single-GPU form; entries of ranks on other GPUs are addresses of PEER memory
+ * mapped into this process (CUDA IPC or symmetric memory), entries the call does not touch may be NULL.  Only ranks
+ * [rank_begin, rank_begin + rank_count) - the ranks this GPU hosts - act:
+ *   basp_reshard_qkv_s2h_ranks  pushes their sequence shards into the head shards of every member of their groups
+ *                               (plain stores; remote members over NVLink);
+ *   basp_attn_fwd_ranks         attention over their own head shards (local memory only);
+ *   basp_reshard_h2s_ranks      pulls their sequence shards of O together from the group's head shards (plain loads);
+ *   basp_layer_fwd_fused_ranks  the three steps as one kernel: Q/K/V tiles are fetched from the group's sequence
+ *                               shards wherever they live (TMA tile loads without multicast) and O tiles are stored
+ *                               into the owner's sequence shard - exchange and attention overlap tile by tile.
+ * The caller orders the GPUs on the host: every GPU's inputs are complete before any GPU launches, and nobody reuses
+ * a buffer before all GPUs' launches have finished (a barrier of the process group on both sides; the kernels never
+ * wait for one another).  The union of the calls over all GPUs equals the single-GPU call bit for bit.
+ * Errors as the single-GPU forms; INVALID for a range outside [0, n_ranks). */
+int basp_reshard_qkv_s2h_ranks(const basp_plan *plan, const void *const *q_seq, const void *const *k_seq,
+                               const void *const *v_seq, void *const *q_head, void *const *k_head,
+                               void *const *v_head, int rank_begin, int rank_count, void *stream);
+int basp_reshard_h2s_ranks(const basp_plan *plan, int n_heads, const void *const *head_shards,
+                           void *const *seq_shards, int rank_begin, int rank_count, void *stream);
+int basp_attn_fwd_ranks(const basp_plan *plan, const void *const *q_head, const void *const *k_head,
+                        const void *const *v_head, void *const *o_head, float *const *lse_shards,
+                        float softmax_scale, int rank_begin, int rank_count, void *stream);
+int basp_layer_fwd_fused_ranks(const basp_plan *plan, const void *const *q_seq, const void *const *k_seq,
+                               const void *const *v_seq, void *const *o_seq, float *const *lse_shards,
+                               float softmax_scale, int rank_begin, int rank_count, void *stream);
+
 /* After basp_layer_fwd (or basp_layer_fwd_static) returns, the workspace holds the head-sharded
  * Q, K, V and O of every rank; this call writes their addresses (n_ranks pointers each) so that a
  * training step can keep them for the backward pass instead of resharding again. */

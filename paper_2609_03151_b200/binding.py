@@ -30,6 +30,7 @@ EXPORTS = [
     "basp_layer_workspace_shards", "basp_attn_bwd", "basp_attn_bwd_workspace_bytes", "basp_reshard_grads_h2s",
     "basp_layer_bwd", "basp_layer_bwd_workspace_bytes", "basp_get_status", "basp_clear_status",
     "basp_strerror", "basp_last_cuda_error", "basp_launch_count", "basp_selftest_wait_timeout", "basp_qkv_proj", "basp_out_proj",
+    "basp_reshard_qkv_s2h_ranks", "basp_reshard_h2s_ranks", "basp_attn_fwd_ranks", "basp_layer_fwd_fused_ranks",
 ]
 
 
@@ -61,6 +62,10 @@ lib.basp_reshard_qkv_s2h.argtypes = [c_void_p] + [_PP] * 6 + [c_void_p]
 lib.basp_attn_fwd.argtypes = [c_void_p] + [_PP] * 5 + [c_float, c_void_p]
 lib.basp_layer_fwd.argtypes = [c_void_p] + [_PP] * 5 + [c_void_p, c_size_t, c_float, c_void_p]
 lib.basp_layer_fwd_fused.argtypes = [c_void_p] + [_PP] * 5 + [c_float, c_void_p]
+lib.basp_reshard_qkv_s2h_ranks.argtypes = [c_void_p] + [_PP] * 6 + [c_int, c_int, c_void_p]
+lib.basp_reshard_h2s_ranks.argtypes = [c_void_p, c_int, _PP, _PP, c_int, c_int, c_void_p]
+lib.basp_attn_fwd_ranks.argtypes = [c_void_p] + [_PP] * 5 + [c_float, c_int, c_int, c_void_p]
+lib.basp_layer_fwd_fused_ranks.argtypes = [c_void_p] + [_PP] * 5 + [c_float, c_int, c_int, c_void_p]
 lib.basp_layer_fwd_static.argtypes = [c_void_p] + [_PP] * 5 + [c_float, c_void_p]
 lib.basp_layer_fwd_host.argtypes = [c_void_p] + [_PP] * 4 + [c_void_p, c_size_t, c_float, c_void_p]
 lib.basp_layer_workspace_shards.argtypes = [c_void_p, c_void_p] + [_PP] * 4
@@ -99,12 +104,14 @@ def _check(code: int, where: str):
 
 
 def _ptrs(tensors, n: int):
-    """Host array of n raw addresses from a list of tensors (or None entries -> NULL)."""
+    """Host array of n raw addresses from a list of tensors, raw integer addresses (peer memory mapped into this
+    process) or None entries (-> NULL)."""
     if tensors is None:
         return None
     if len(tensors) != n:
         raise ValueError(f"expected {n} shards, got {len(tensors)}")
-    return (c_void_p * n)(*[None if t is None else t.data_ptr() for t in tensors])
+    return (c_void_p * n)(*[None if t is None else (t.data_ptr() if hasattr(t, "data_ptr") else int(t))
+                            for t in tensors])
 
 
 def _stream(stream):
@@ -197,6 +204,37 @@ def basp_layer_fwd_fused(plan, q_seq, k_seq, v_seq, o_seq, lse_shards=None, soft
     _check(lib.basp_layer_fwd_fused(plan.handle, _ptrs(q_seq, n), _ptrs(k_seq, n), _ptrs(v_seq, n),
                                     _ptrs(o_seq, n), _ptrs(lse_shards, n), softmax_scale, _stream(stream)),
            "basp_layer_fwd_fused")
+
+
+# ---- one physical GPU's share (ranks [rank_begin, rank_begin + rank_count)); shard lists may hold tensors, raw
+# addresses of peer memory, or None for shards the call does not touch
+def basp_reshard_qkv_s2h_ranks(plan, q_seq, k_seq, v_seq, q_head, k_head, v_head, rank_begin, rank_count, stream=None):
+    n = plan.N
+    _check(lib.basp_reshard_qkv_s2h_ranks(plan.handle, _ptrs(q_seq, n), _ptrs(k_seq, n), _ptrs(v_seq, n),
+                                          _ptrs(q_head, n), _ptrs(k_head, n), _ptrs(v_head, n), rank_begin,
+                                          rank_count, _stream(stream)), "basp_reshard_qkv_s2h_ranks")
+
+
+def basp_reshard_h2s_ranks(plan, n_heads, head_shards, seq_shards, rank_begin, rank_count, stream=None):
+    n = plan.N
+    _check(lib.basp_reshard_h2s_ranks(plan.handle, n_heads, _ptrs(head_shards, n), _ptrs(seq_shards, n), rank_begin,
+                                      rank_count, _stream(stream)), "basp_reshard_h2s_ranks")
+
+
+def basp_attn_fwd_ranks(plan, q_head, k_head, v_head, o_head, rank_begin, rank_count, lse_shards=None,
+                        softmax_scale=0.0, stream=None):
+    n = plan.N
+    _check(lib.basp_attn_fwd_ranks(plan.handle, _ptrs(q_head, n), _ptrs(k_head, n), _ptrs(v_head, n),
+                                   _ptrs(o_head, n), _ptrs(lse_shards, n), softmax_scale, rank_begin, rank_count,
+                                   _stream(stream)), "basp_attn_fwd_ranks")
+
+
+def basp_layer_fwd_fused_ranks(plan, q_seq, k_seq, v_seq, o_seq, rank_begin, rank_count, lse_shards=None,
+                               softmax_scale=0.0, stream=None):
+    n = plan.N
+    _check(lib.basp_layer_fwd_fused_ranks(plan.handle, _ptrs(q_seq, n), _ptrs(k_seq, n), _ptrs(v_seq, n),
+                                          _ptrs(o_seq, n), _ptrs(lse_shards, n), softmax_scale, rank_begin,
+                                          rank_count, _stream(stream)), "basp_layer_fwd_fused_ranks")
 
 
 BASP_STATIC_SCRATCH_BYTES = 16 << 20

@@ -38,7 +38,11 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
     AttnParams<R> prm;
     const uint64_t rows = (uint64_t)pl->Bl * (fused ? pl->T : pl->S);
     const int hq = fused ? pl->Hq : pl->Hq_l, hkv = fused ? pl->Hkv : pl->Hkv_l;
-    for (int r = 0; r < pl->N; ++r) {
+    // Operands of ranks outside the launch's range are not touched: with head-sharded operands only the ranks of the
+    // range, with sequence-sharded (fused) operands every member of their groups.
+    const int need_lo = fused ? range[0] / pl->K * pl->K : range[0];
+    const int need_hi = fused ? (range[0] + range[1] + pl->K - 1) / pl->K * pl->K : range[0] + range[1];
+    for (int r = need_lo; r < need_hi; ++r) {
         int rc = tmap::encode_rows_heads_d(&prm.q[r], q[r], rows, hq, pl->D, kTile);
         if (rc == BASP_OK) rc = tmap::encode_rows_heads_d(&prm.k[r], k[r], rows, hkv, pl->D, kTile);
         if (rc == BASP_OK) rc = tmap::encode_rows_heads_d(&prm.v[r], v[r], rows, hkv, pl->D, kTile);
@@ -93,16 +97,21 @@ int basp_attn_dispatch_range(const basp_plan *pl, const void *const *q, const vo
     if (!pl || !q || !k || !v || !o) return BASP_ERR_NULL;
     if (pl->D != 64 && pl->D != 128) return BASP_ERR_UNSUPPORTED;
     if (fused && pl->T % kTile != 0) return BASP_ERR_UNSUPPORTED;
-    for (int r = 0; r < pl->N; ++r) {
-        if (!q[r] || !k[r] || !v[r] || !o[r] || (lse && !lse[r])) return BASP_ERR_NULL;
-        if (!aligned16(q[r]) || !aligned16(k[r]) || !aligned16(v[r]) || !aligned16(o[r]) || (lse && ((uintptr_t)lse[r] & 3)))
-            return BASP_ERR_ALIGN;
-        for (int r2 = 0; r2 < pl->N; ++r2)
-            if (o[r] == q[r2] || o[r] == k[r2] || o[r] == v[r2]) return BASP_ERR_ALIAS;
-    }
     const int full[4] = {0, pl->N, 0, ((pl->S + kTile - 1) / kTile + 1) / 2};
     if (!range) range = full;
+    if (range[0] < 0 || range[1] < 0 || range[0] + range[1] > pl->N) return BASP_ERR_INVALID;
     if (range[1] <= 0 || range[3] <= 0) return BASP_OK;
+    const int need_lo = fused ? range[0] / pl->K * pl->K : range[0];
+    const int need_hi = fused ? (range[0] + range[1] + pl->K - 1) / pl->K * pl->K : range[0] + range[1];
+    for (int r = need_lo; r < need_hi; ++r) {
+        const bool own = r >= range[0] && r < range[0] + range[1];       // LSE is written by the ranks of the range only
+        if (!q[r] || !k[r] || !v[r] || !o[r] || (lse && own && !lse[r])) return BASP_ERR_NULL;
+        if (!aligned16(q[r]) || !aligned16(k[r]) || !aligned16(v[r]) || !aligned16(o[r]) ||
+            (lse && own && ((uintptr_t)lse[r] & 3)))
+            return BASP_ERR_ALIGN;
+        for (int r2 = need_lo; r2 < need_hi; ++r2)
+            if (o[r] == q[r2] || o[r] == k[r2] || o[r] == v[r2]) return BASP_ERR_ALIAS;
+    }
     if (pl->N <= 8) return fill_and_launch<8>(pl, q, k, v, o, lse, scale, fused, range, (cudaStream_t)stream);
     return fill_and_launch<BASP_MAX_RANKS>(pl, q, k, v, o, lse, scale, fused, range, (cudaStream_t)stream);
 }
@@ -122,4 +131,25 @@ extern "C" int basp_layer_fwd_fused(const basp_plan *plan, const void *const *q_
                                     const void *const *v_seq, void *const *o_seq, float *const *lse_shards,
                                     float softmax_scale, void *stream) {
     return basp_attn_dispatch(plan, q_seq, k_seq, v_seq, o_seq, lse_shards, softmax_scale, true, stream);
+}
+
+// One physical GPU's share when the N ranks are spread over several GPUs: only ranks [rank_begin, rank_begin +
+// rank_count) compute.  Head-sharded operands of other ranks are not touched.  With sequence-sharded operands (fused)
+// the tiles of the other members of the range's groups are fetched from wherever their pointers lead - peer memory
+// mapped into this process included (plain TMA tile loads, no multicast) - and O tiles are stored there with plain
+// stores: the all-to-alls of Section IV-C and the attention in one kernel over NVLink.
+extern "C" int basp_attn_fwd_ranks(const basp_plan *plan, const void *const *q_head, const void *const *k_head,
+                                   const void *const *v_head, void *const *o_head, float *const *lse_shards,
+                                   float softmax_scale, int rank_begin, int rank_count, void *stream) {
+    if (!plan) return BASP_ERR_NULL;
+    const int range[4] = {rank_begin, rank_count, 0, ((plan->S + kTile - 1) / kTile + 1) / 2};
+    return basp_attn_dispatch_range(plan, q_head, k_head, v_head, o_head, lse_shards, softmax_scale, false, range, stream);
+}
+
+extern "C" int basp_layer_fwd_fused_ranks(const basp_plan *plan, const void *const *q_seq, const void *const *k_seq,
+                                          const void *const *v_seq, void *const *o_seq, float *const *lse_shards,
+                                          float softmax_scale, int rank_begin, int rank_count, void *stream) {
+    if (!plan) return BASP_ERR_NULL;
+    const int range[4] = {rank_begin, rank_count, 0, ((plan->S + kTile - 1) / kTile + 1) / 2};
+    return basp_attn_dispatch_range(plan, q_seq, k_seq, v_seq, o_seq, lse_shards, softmax_scale, true, range, stream);
 }

@@ -33,6 +33,7 @@ struct ReshardTensor {
 
 struct ReshardParams {
     int n_tensors;
+    uint32_t r_begin, r_count; // sequence-side ranks this launch walks
     uint32_t K, T, S;
     FastDiv div_T;
     ReshardTensor t[3];
@@ -58,8 +59,9 @@ __global__ void __launch_bounds__(kThreads) reshard_kernel(const __grid_constant
     while (ti + 1 < p.n_tensors && c >= p.t[ti + 1].chunk_begin) ++ti;
     const ReshardTensor &t = p.t[ti];
     c -= t.chunk_begin;
-    const uint32_t r = c / t.chunks_per_shard;
-    const uint32_t chunk = c - r * t.chunks_per_shard;
+    const uint32_t ri = c / t.chunks_per_shard;
+    const uint32_t chunk = c - ri * t.chunks_per_shard;
+    const uint32_t r = p.r_begin + ri;
     const uint32_t g = r / p.K, l = r - g * p.K;
     const uint32_t v0 = chunk * kChunkV + threadIdx.x;
 
@@ -97,25 +99,28 @@ struct TensorArg {
     const void *const *head;
 };
 
-int fill_tensor(const basp_plan *p, const TensorArg &a, bool to_head, ReshardTensor *t, uint32_t *chunk_cursor) {
+int fill_tensor(const basp_plan *p, const TensorArg &a, bool to_head, int r_begin, int r_count, ReshardTensor *t,
+                uint32_t *chunk_cursor) {
     if (!a.seq || !a.head) return BASP_ERR_NULL;
     if (a.n_heads <= 0 || a.n_heads % p->K != 0) return BASP_ERR_INVALID;
     const size_t run_bytes = (size_t)(a.n_heads / p->K) * p->D * 2;
     if (run_bytes % 16 != 0) return BASP_ERR_UNSUPPORTED;
     const size_t shard_bytes = (size_t)p->Bl * p->T * a.n_heads * p->D * 2;
     if (shard_bytes / 16 >= (1ull << 31)) return BASP_ERR_UNSUPPORTED;
+    // The launch walks the sequence-side shards of ranks [r_begin, r_begin + r_count) and touches the head-side
+    // shards of every member of their groups; the other entries are not read (they may be NULL).
+    const int g_begin = r_begin / p->K * p->K, g_end = (r_begin + r_count + p->K - 1) / p->K * p->K;
     for (int r = 0; r < p->N; ++r) {
-        if (!a.seq[r] || !a.head[r]) return BASP_ERR_NULL;
-        if (!aligned16(a.seq[r]) || !aligned16(a.head[r])) return BASP_ERR_ALIGN;
-        t->seq[r] = (const char *)a.seq[r];
-        t->head[r] = (const char *)a.head[r];
+        const bool need_seq = r >= r_begin && r < r_begin + r_count, need_head = r >= g_begin && r < g_end;
+        t->seq[r] = need_seq ? (const char *)a.seq[r] : nullptr;
+        t->head[r] = need_head ? (const char *)a.head[r] : nullptr;
+        if ((need_seq && !a.seq[r]) || (need_head && !a.head[r])) return BASP_ERR_NULL;
+        if ((need_seq && !aligned16(a.seq[r])) || (need_head && !aligned16(a.head[r]))) return BASP_ERR_ALIGN;
     }
     // out-of-place only: no destination shard may overlap a source shard
-    const void *const *src = to_head ? a.seq : a.head;
-    const void *const *dst = to_head ? a.head : a.seq;
-    for (int i = 0; i < p->N; ++i)
-        for (int j = 0; j < p->N; ++j) {
-            const char *s = (const char *)src[i], *d = (const char *)dst[j];
+    for (int i = r_begin; i < r_begin + r_count; ++i)
+        for (int j = g_begin; j < g_end; ++j) {
+            const char *s = t->seq[i], *d = t->head[j];
             if (s < d + shard_bytes && d < s + shard_bytes) return BASP_ERR_ALIAS;
         }
     t->run_v = (uint32_t)(run_bytes / 16);
@@ -125,19 +130,23 @@ int fill_tensor(const basp_plan *p, const TensorArg &a, bool to_head, ReshardTen
     t->chunk_begin = *chunk_cursor;
     t->div_row = make_fastdiv(t->row_v);
     t->div_run = make_fastdiv(t->run_v);
-    *chunk_cursor += t->chunks_per_shard * (uint32_t)p->N;
+    *chunk_cursor += t->chunks_per_shard * (uint32_t)r_count;
     return BASP_OK;
 }
 
-int launch(const basp_plan *p, const TensorArg *args, int n, bool to_head, void *stream) {
+int launch(const basp_plan *p, const TensorArg *args, int n, bool to_head, int r_begin, int r_count, void *stream) {
     if (!p) return BASP_ERR_NULL;
+    if (r_count < 0) { r_begin = 0; r_count = p->N; }          // every rank
+    if (r_begin < 0 || r_begin + r_count > p->N) return BASP_ERR_INVALID;
+    if (r_count == 0) return BASP_OK;
     ReshardParams prm;
     prm.n_tensors = n;
+    prm.r_begin = (uint32_t)r_begin; prm.r_count = (uint32_t)r_count;
     prm.K = p->K; prm.T = p->T; prm.S = p->S;
     prm.div_T = make_fastdiv((uint32_t)p->T);
     uint32_t chunks = 0;
     for (int i = 0; i < n; ++i) {
-        int rc = fill_tensor(p, args[i], to_head, &prm.t[i], &chunks);
+        int rc = fill_tensor(p, args[i], to_head, r_begin, r_count, &prm.t[i], &chunks);
         if (rc != BASP_OK) return rc;
     }
     if (chunks == 0) return BASP_OK;
@@ -154,13 +163,13 @@ int launch(const basp_plan *p, const TensorArg *args, int n, bool to_head, void 
 extern "C" int basp_reshard_s2h(const basp_plan *plan, int n_heads, const void *const *seq_shards,
                                 void *const *head_shards, void *stream) {
     TensorArg a{n_heads, seq_shards, (const void *const *)head_shards};
-    return launch(plan, &a, 1, true, stream);
+    return launch(plan, &a, 1, true, 0, -1, stream);
 }
 
 extern "C" int basp_reshard_h2s(const basp_plan *plan, int n_heads, const void *const *head_shards,
                                 void *const *seq_shards, void *stream) {
     TensorArg a{n_heads, (const void *const *)seq_shards, head_shards};
-    return launch(plan, &a, 1, false, stream);
+    return launch(plan, &a, 1, false, 0, -1, stream);
 }
 
 extern "C" int basp_reshard_qkv_s2h(const basp_plan *plan, const void *const *q_seq,
@@ -171,7 +180,7 @@ extern "C" int basp_reshard_qkv_s2h(const basp_plan *plan, const void *const *q_
     TensorArg a[3] = {{plan->Hq, q_seq, (const void *const *)q_head},
                       {plan->Hkv, k_seq, (const void *const *)k_head},
                       {plan->Hkv, v_seq, (const void *const *)v_head}};
-    return launch(plan, a, 3, true, stream);
+    return launch(plan, a, 3, true, 0, -1, stream);
 }
 
 extern "C" int basp_reshard_grads_h2s(const basp_plan *plan, const void *const *dq_head, const void *const *dk_head,
@@ -181,5 +190,26 @@ extern "C" int basp_reshard_grads_h2s(const basp_plan *plan, const void *const *
     TensorArg a[3] = {{plan->Hq, (const void *const *)dq_seq, dq_head},
                       {plan->Hkv, (const void *const *)dk_seq, dk_head},
                       {plan->Hkv, (const void *const *)dv_seq, dv_head}};
-    return launch(plan, a, 3, false, stream);
+    return launch(plan, a, 3, false, 0, -1, stream);
+}
+
+// The same exchanges restricted to the sequence-side shards of ranks [rank_begin, rank_begin + rank_count): what ONE
+// physical GPU launches when a group spans several GPUs and the other ranks' shards are peer memory.  s2h pushes
+// this GPU's sequence shards into every group member's head shard; h2s pulls this GPU's sequence shards together.
+extern "C" int basp_reshard_qkv_s2h_ranks(const basp_plan *plan, const void *const *q_seq, const void *const *k_seq,
+                                          const void *const *v_seq, void *const *q_head, void *const *k_head,
+                                          void *const *v_head, int rank_begin, int rank_count, void *stream) {
+    if (!plan) return BASP_ERR_NULL;
+    if (rank_count < 0) return BASP_ERR_INVALID;
+    TensorArg a[3] = {{plan->Hq, q_seq, (const void *const *)q_head},
+                      {plan->Hkv, k_seq, (const void *const *)k_head},
+                      {plan->Hkv, v_seq, (const void *const *)v_head}};
+    return launch(plan, a, 3, true, rank_begin, rank_count, stream);
+}
+
+extern "C" int basp_reshard_h2s_ranks(const basp_plan *plan, int n_heads, const void *const *head_shards,
+                                      void *const *seq_shards, int rank_begin, int rank_count, void *stream) {
+    if (rank_count < 0) return BASP_ERR_INVALID;
+    TensorArg a{n_heads, (const void *const *)seq_shards, head_shards};
+    return launch(plan, &a, 1, false, rank_begin, rank_count, stream);
 }

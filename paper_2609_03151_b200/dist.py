@@ -3,6 +3,11 @@
 The path shards without any data-path collective: BASP groups are independent units (each
 group's all-to-all stays inside the group), so different GPUs take different groups -- or,
 for weak scaling, different micro-batches -- and only timing is reduced across ranks.
+
+When a group does span GPUs (K > N / world) the exchange is real: every GPU then runs the
+`*_ranks` calls for the ranks it hosts over shard tables that point into its peers' memory
+(`SymmetricShards`, `layer_fwd_fused_multi_gpu`); the kernels use plain loads/stores and TMA tile
+loads without multicast on that memory and never wait for one another.
 """
 from __future__ import annotations
 
@@ -66,6 +71,80 @@ def groups_of_gpu(num_groups: int, world: int, rank: int) -> range:
                          "(a group split across GPUs would need a real all-to-all)")
     per = num_groups // world
     return range(rank * per, (rank + 1) * per)
+
+
+def ranks_of_gpu(n_ranks: int, world: int, gpu: int) -> range:
+    """The contiguous block of virtual ranks that physical GPU `gpu` of `world` hosts (rank r lives on GPU
+    floor(r * world / N), Section IV-A).  Needs world to divide n_ranks.  A group (K consecutive ranks) then lies on
+    one GPU when K <= N / world and otherwise spans K * world / N GPUs."""
+    if world <= 0 or n_ranks % world != 0:
+        raise ValueError("the number of GPUs must divide the number of ranks")
+    per = n_ranks // world
+    if not 0 <= gpu < world:
+        raise ValueError("gpu out of range")
+    return range(gpu * per, (gpu + 1) * per)
+
+
+def gpu_of_rank(n_ranks: int, world: int, rank: int) -> int:
+    return rank // (n_ranks // world)
+
+
+def shard_addresses(buffer_ptrs, n_ranks: int, shard_bytes: int, offset: int = 0) -> list[int]:
+    """Addresses, valid in THIS process, of every rank's shard of one tensor when each GPU keeps the shards of its
+    ranks back to back in one symmetric buffer: `buffer_ptrs[g]` is the address at which GPU g's buffer is mapped
+    here (the local allocation for g = this GPU, peer memory otherwise), `offset` the tensor's byte offset inside
+    every buffer.  The result is what the `*_ranks` calls take as their shard arrays."""
+    world = len(buffer_ptrs)
+    per = len(ranks_of_gpu(n_ranks, world, 0))
+    if offset % 16 or shard_bytes % 16:
+        raise ValueError("shards must stay 16-byte aligned")
+    return [int(buffer_ptrs[r // per]) + offset + (r % per) * shard_bytes for r in range(n_ranks)]
+
+
+class SymmetricShards:
+    """One symmetric-memory buffer per GPU holding this GPU's shards of several tensors, mapped into every process of
+    the group (torch symmetric memory over NVLink).  `tensors` = {name: shard_bytes}.  Needs an initialised NCCL
+    process group with one process per GPU."""
+
+    def __init__(self, n_ranks: int, tensors: dict, group=None):
+        import torch.distributed._symmetric_memory as symm_mem
+        self.group = group if group is not None else dist.group.WORLD
+        self.world, self.gpu = dist.get_world_size(self.group), dist.get_rank(self.group)
+        self.n_ranks, self.local = n_ranks, ranks_of_gpu(n_ranks, self.world, self.gpu)
+        self.layout, off = {}, 0
+        for name, shard_bytes in tensors.items():
+            self.layout[name] = (off, int(shard_bytes))
+            off += (len(self.local) * int(shard_bytes) + 255) // 256 * 256
+        self.buffer = symm_mem.empty(off, dtype=torch.uint8, device=torch.device("cuda", torch.cuda.current_device()))
+        self.handle = symm_mem.rendezvous(self.buffer, self.group)
+        self.buffer_ptrs = [int(p) for p in self.handle.buffer_ptrs]
+
+    def addresses(self, name: str) -> list[int]:
+        off, shard_bytes = self.layout[name]
+        return shard_addresses(self.buffer_ptrs, self.n_ranks, shard_bytes, off)
+
+    def local_shard(self, name: str, rank: int) -> torch.Tensor:
+        """This GPU's shard of rank `rank` as a byte tensor (view it as bf16 and reshape)."""
+        off, shard_bytes = self.layout[name]
+        i = rank - self.local.start
+        if not 0 <= i < len(self.local):
+            raise ValueError("rank lives on another GPU")
+        return self.buffer[off + i * shard_bytes: off + (i + 1) * shard_bytes]
+
+
+def layer_fwd_fused_multi_gpu(plan, shards: "SymmetricShards", softmax_scale: float = 0.0, stream=None):
+    """The layer when a group spans GPUs: every GPU runs the fused kernel for its own ranks over the group's
+    sequence shards (`shards` holds tensors "q", "k", "v", "o").  The kernels never wait for one another: the two
+    host barriers order the GPUs (inputs complete before anyone reads them, nobody reuses a buffer before all are
+    done)."""
+    from . import binding
+    torch.cuda.current_stream().synchronize()
+    dist.barrier(shards.group)
+    binding.basp_layer_fwd_fused_ranks(plan, shards.addresses("q"), shards.addresses("k"), shards.addresses("v"),
+                                       shards.addresses("o"), shards.local.start, len(shards.local),
+                                       softmax_scale=softmax_scale, stream=stream)
+    torch.cuda.current_stream().synchronize()
+    dist.barrier(shards.group)
 
 
 def finalize():

@@ -60,3 +60,65 @@ def test_groups_of_gpu():
         assert False
     except ValueError:
         pass
+
+
+def _worker_span(rank, world, port, out_dir):
+    """A group that spans both processes (K = 4 ranks on 2 'GPUs'): address tables and the push exchange."""
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    pdist.init(backend="gloo")
+    wl = synth.Workload("g", N=4, B=1, S=64, Hq=4, Hkv=4, D=8)
+    Xq, _, _ = (synth.bits(t) for t in synth.make_qkv(wl, seed=1))
+    pl = oracle.plan(wl.N, wl.B, wl.S)
+    mine = pdist.ranks_of_gpu(wl.N, world, rank)
+    assert len(mine) == 2 and pdist.gpu_of_rank(wl.N, world, mine.start) == rank
+    # every process publishes where its buffer is "mapped": the tables built from the gathered bases must agree
+    shard_bytes = pl.Bl * pl.T * wl.Hq * wl.D * 2
+    bases = [None] * world
+    dist.all_gather_object(bases, 0x10000000 * (rank + 1))
+    table = pdist.shard_addresses(bases, wl.N, shard_bytes, offset=256)
+    assert table == [0x10000000 * (r // 2 + 1) + 256 + (r % 2) * shard_bytes for r in range(wl.N)]
+    tables = [None] * world
+    dist.all_gather_object(tables, table)
+    assert tables[0] == tables[1]
+    # push model of the s2h exchange: every process scatters only ITS ranks' sequence shards; the pieces are disjoint
+    # and their union is the whole exchange
+    seq = oracle.partition(Xq, pl)
+    masked = seq.copy()
+    for r in range(wl.N):
+        if r not in mine:
+            masked[r] = 0
+    part = oracle.s2h(masked, pl).astype(np.int64)
+    total = torch.from_numpy(part.copy())
+    dist.all_reduce(total, op=dist.ReduceOp.SUM)
+    full = oracle.s2h(seq, pl).astype(np.int64)
+    assert np.array_equal(total.numpy(), full)
+    nz = torch.from_numpy((part != 0).astype(np.int64))
+    dist.all_reduce(nz, op=dist.ReduceOp.SUM)
+    assert int(nz.max()) <= 1                      # no element written by two processes
+    pdist.finalize()
+    open(os.path.join(out_dir, f"span{rank}"), "w").write("ok")
+
+
+def test_two_process_group_spanning_exchange(tmp_path):
+    port = _free_port()
+    mp.spawn(_worker_span, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    assert all((tmp_path / f"span{r}").exists() for r in range(2))
+
+
+def test_ranks_of_gpu_and_addresses():
+    assert list(pdist.ranks_of_gpu(8, 2, 1)) == [4, 5, 6, 7]
+    assert list(pdist.ranks_of_gpu(8, 8, 3)) == [3]
+    assert [pdist.gpu_of_rank(8, 4, r) for r in range(8)] == [0, 0, 1, 1, 2, 2, 3, 3]
+    for bad in ((8, 3, 0), (8, 2, 2)):
+        try:
+            pdist.ranks_of_gpu(*bad)
+            assert False
+        except ValueError:
+            pass
+    assert pdist.shard_addresses([1000 * 16, 5000 * 16], 4, 32) == [16000, 16032, 80000, 80032]
+    try:
+        pdist.shard_addresses([0, 0], 4, 24)
+        assert False
+    except ValueError:
+        pass
