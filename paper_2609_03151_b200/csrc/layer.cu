@@ -95,6 +95,7 @@ namespace {
 struct HostPipe {
     cudaStream_t in = nullptr, out = nullptr;
     cudaEvent_t start = nullptr, done = nullptr, arrived[BASP_MAX_RANKS] = {}, computed[BASP_MAX_RANKS] = {};
+    cudaEvent_t kv_arrived[BASP_MAX_RANKS] = {};   // per group
 };
 std::mutex g_pipe_mu;
 HostPipe g_pipes[64];
@@ -113,6 +114,7 @@ int get_pipe(HostPipe **out) {
         for (int i = 0; i < BASP_MAX_RANKS; ++i) {
             BASP_CUDA_TRY(cudaEventCreateWithFlags(&p.arrived[i], cudaEventDisableTiming));
             BASP_CUDA_TRY(cudaEventCreateWithFlags(&p.computed[i], cudaEventDisableTiming));
+            BASP_CUDA_TRY(cudaEventCreateWithFlags(&p.kv_arrived[i], cudaEventDisableTiming));
         }
     }
     *out = &p;
@@ -120,10 +122,12 @@ int get_pipe(HostPipe **out) {
 }
 }  // namespace
 
-// Copies, kernels and read-backs are pipelined.  With the causal mask the query rows that local rank l
-// owns only need the shards of local ranks 0..l of its group, so the launch for those rows starts as soon
-// as shard l has arrived while later shards are still on the bus, and O shard l is read back as soon as
-// that launch is done (three streams: copies in, the caller's stream for the kernels, copies out).
+// Copies, kernels and read-backs are pipelined (three streams: copies in, the caller's stream for the kernels,
+// copies out).  The bus is the slow part, so the order of the copies is chosen to give the GPU its longest work
+// first: per group the K and V shards (a quarter of the bytes under GQA) go first, then the Q shards from the LAST
+// local rank down.  Under the causal mask the rows of local rank l cost (2l+1)/K^2 of the group's arithmetic, so
+// the launch for the last rank's rows - the longest - starts after K, V and one Q shard have arrived and the
+// shorter ones follow while the rest is still on the bus; O shard l is read back as soon as its launch is done.
 // Calls that overlap in time on one device share the internal streams and events: serialise them.
 extern "C" int basp_layer_fwd_host(const basp_plan *p, const void *const *q_seq_host, const void *const *k_seq_host,
                                    const void *const *v_seq_host, void *const *o_seq_host, void *device_arena,
@@ -149,16 +153,23 @@ extern "C" int basp_layer_fwd_host(const basp_plan *p, const void *const *q_seq_
     BASP_CUDA_TRY(cudaEventRecord(pipe->start, st));
     BASP_CUDA_TRY(cudaStreamWaitEvent(pipe->in, pipe->start, 0));
     BASP_CUDA_TRY(cudaStreamWaitEvent(pipe->out, pipe->start, 0));
-    for (int r = 0; r < p->N; ++r) {
-        BASP_CUDA_TRY(cudaMemcpyAsync(kd[r], k_seq_host[r], kb, cudaMemcpyHostToDevice, pipe->in));
-        BASP_CUDA_TRY(cudaMemcpyAsync(vd[r], v_seq_host[r], kb, cudaMemcpyHostToDevice, pipe->in));
-        BASP_CUDA_TRY(cudaMemcpyAsync(qd[r], q_seq_host[r], qb, cudaMemcpyHostToDevice, pipe->in));
-        BASP_CUDA_TRY(cudaEventRecord(pipe->arrived[r], pipe->in));
+    for (int g = 0; g < p->G; ++g) {
+        const int r0 = g * p->K;
+        for (int l = 0; l < p->K; ++l) {
+            BASP_CUDA_TRY(cudaMemcpyAsync(kd[r0 + l], k_seq_host[r0 + l], kb, cudaMemcpyHostToDevice, pipe->in));
+            BASP_CUDA_TRY(cudaMemcpyAsync(vd[r0 + l], v_seq_host[r0 + l], kb, cudaMemcpyHostToDevice, pipe->in));
+        }
+        BASP_CUDA_TRY(cudaEventRecord(pipe->kv_arrived[g], pipe->in));
+        for (int l = p->K - 1; l >= 0; --l) {
+            BASP_CUDA_TRY(cudaMemcpyAsync(qd[r0 + l], q_seq_host[r0 + l], qb, cudaMemcpyHostToDevice, pipe->in));
+            BASP_CUDA_TRY(cudaEventRecord(pipe->arrived[r0 + l], pipe->in));
+        }
     }
     for (int g = 0; g < p->G; ++g) {
         const int r0 = g * p->K;
+        BASP_CUDA_TRY(cudaStreamWaitEvent(st, pipe->kv_arrived[g], 0));
         if (by_chunk) {
-            for (int l = 0; l < p->K; ++l) {
+            for (int l = p->K - 1; l >= 0; --l) {
                 BASP_CUDA_TRY(cudaStreamWaitEvent(st, pipe->arrived[r0 + l], 0));
                 const int range[4] = {r0, p->K, l * (p->T / 256), p->T / 256};
                 rc = basp_attn_dispatch_range(p, qd, kd, vd, od, nullptr, softmax_scale, true, range, stream);
@@ -168,7 +179,7 @@ extern "C" int basp_layer_fwd_host(const basp_plan *p, const void *const *q_seq_
                 BASP_CUDA_TRY(cudaMemcpyAsync(o_seq_host[r0 + l], od[r0 + l], qb, cudaMemcpyDeviceToHost, pipe->out));
             }
         } else {
-            BASP_CUDA_TRY(cudaStreamWaitEvent(st, pipe->arrived[r0 + p->K - 1], 0));
+            BASP_CUDA_TRY(cudaStreamWaitEvent(st, pipe->arrived[r0], 0));      // the Q shard sent last
             const int range[4] = {r0, p->K, 0, (p->S / 128 + 1) / 2};
             rc = basp_attn_dispatch_range(p, qd, kd, vd, od, nullptr, softmax_scale, true, range, stream);
             if (rc != BASP_OK) return rc;
