@@ -127,7 +127,8 @@ int basp_reshard_qkv_s2h(const basp_plan *plan, const void *const *q_seq, const 
  * Inputs/outputs are HEAD-sharded; lse_shards may be NULL (then no LSE is written), else a
  * host array of n_ranks device pointers to fp32 [Bl][Hq/K][S].  softmax_scale = 0 selects
  * 1/sqrt(D).  bf16 operands, fp32 accumulation and softmax, P rounded to bf16 before P.V.
- * Requires D in {64, 128} (else BASP_ERR_UNSUPPORTED); S is arbitrary (a ragged last tile is masked).
+ * Requires D a multiple of 16 up to 128 (else BASP_ERR_UNSUPPORTED; the kernels are 64 and 128 columns wide, for a
+ * D in between the tile loads zero-fill the missing columns); S is arbitrary (a ragged last tile is masked).
  * A bounded wait that expires inside the kernel is reported by basp_get_status. */
 int basp_attn_fwd(const basp_plan *plan, const void *const *q_head, const void *const *k_head,
                   const void *const *v_head, void *const *o_head, float *const *lse_shards,

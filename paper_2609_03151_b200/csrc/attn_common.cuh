@@ -19,6 +19,8 @@ struct AttnParams {
     float *lse[R];
     int n_ranks, K, Bl, S, T, Hq_l, Hkv_l, q_per_kv;
     int o_heads;            // heads in one row of the O destination (Hq_l, or Hq when fused)
+    int Dg;                 // head dimension in memory, a multiple of 16 up to the kernel's width (64 or 128): the tile
+                            // loads zero-fill the columns past it, the products skip them, the epilogue does not store them
     int qb_band;            // query blocks per scheduling band (divides qb_count)
     int r_begin, r_count;   // ranks covered by this launch
     int qb_begin, qb_count; // 256-row query blocks covered by this launch

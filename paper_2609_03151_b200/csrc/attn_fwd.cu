@@ -53,6 +53,7 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
     prm.n_ranks = pl->N; prm.K = pl->K; prm.Bl = pl->Bl; prm.S = pl->S; prm.T = pl->T;
     prm.Hq_l = pl->Hq_l; prm.Hkv_l = pl->Hkv_l; prm.q_per_kv = pl->Hq / pl->Hkv;
     prm.o_heads = hq;
+    prm.Dg = pl->D;
     {
         const int q_per_kv = pl->Hq / pl->Hkv;
         prm.r_begin = range[0]; prm.r_count = range[1]; prm.qb_begin = range[2]; prm.qb_count = range[3];
@@ -71,7 +72,7 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
         BASP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
         const long long items = (long long)range[3] * range[1] * pl->Bl * pl->Hq_l;
         const int grid = (int)(items < sms ? items : sms);
-        if (pl->D == 128) {
+        if (pl->D > 64) {        // 80 .. 128: the 128-wide kernel
             const int smem = (2 + kStages) * kTile * 128 * 2 + 1024;
             BASP_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_ws_kernel<128, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
             attn_fwd_ws_kernel<128, R><<<grid, kWsThreads, smem, st>>>(prm);
@@ -95,7 +96,7 @@ int basp_attn_dispatch_range(const basp_plan *pl, const void *const *q, const vo
                              void *const *o, float *const *lse, float scale, bool fused, const int *range,
                              void *stream) {
     if (!pl || !q || !k || !v || !o) return BASP_ERR_NULL;
-    if (pl->D != 64 && pl->D != 128) return BASP_ERR_UNSUPPORTED;
+    if (pl->D < 16 || pl->D > 128 || pl->D % 16 != 0) return BASP_ERR_UNSUPPORTED;
     if (fused && pl->T % kTile != 0) return BASP_ERR_UNSUPPORTED;
     const int full[4] = {0, pl->N, 0, ((pl->S + kTile - 1) / kTile + 1) / 2};
     if (!range) range = full;

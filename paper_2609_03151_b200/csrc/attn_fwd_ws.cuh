@@ -322,11 +322,12 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 ++ep_cnt[t];
                 tc_fence_after();
                 const TileCoord c = locate(p, item.r, item.bl, (2 * item.qb + t) * kTile, item.h, p.Hq_l);
-                __nv_bfloat16 *dst = p.o[c.rank] + ((size_t)(c.row + row) * p.o_heads + c.head) * D;
+                __nv_bfloat16 *dst = p.o[c.rank] + ((size_t)(c.row + row) * p.o_heads + c.head) * p.Dg;
                 const uint32_t O_t = tmem + 256 + 128 * t + lane_addr;
                 const bool in_seq = (2 * item.qb + t) * kTile + row < p.S;   // rows past a ragged end are not stored
 #pragma unroll
                 for (int cc = 0; cc < kOCols / 32; ++cc) {
+                    if (cc * 32 >= p.Dg) break;          // columns past the real head dimension are zero padding
                     uint32_t rr[32];
                     tmem_ld_x32(O_t + cc * 32, rr);
                     tmem_wait_ld();
@@ -337,7 +338,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                         o4.y = pack_bf16x2(__uint_as_float(rr[8 * i + 2]) * inv_l, __uint_as_float(rr[8 * i + 3]) * inv_l);
                         o4.z = pack_bf16x2(__uint_as_float(rr[8 * i + 4]) * inv_l, __uint_as_float(rr[8 * i + 5]) * inv_l);
                         o4.w = pack_bf16x2(__uint_as_float(rr[8 * i + 6]) * inv_l, __uint_as_float(rr[8 * i + 7]) * inv_l);
-                        if (in_seq) *reinterpret_cast<uint4 *>(dst + cc * 32 + i * 8) = o4;
+                        if (in_seq && cc * 32 + i * 8 < p.Dg) *reinterpret_cast<uint4 *>(dst + cc * 32 + i * 8) = o4;
                     }
                 }
                 tc_fence_before();
@@ -410,6 +411,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                         if (lane == 0) {
 #pragma unroll
                             for (int kk = 0; kk < D / 16; ++kk) {
+                                if (kk * 16 >= p.Dg) break;   // zero padding contributes nothing to Q.K^T
                                 const uint32_t off16 = ((kk / 4) * 16384 + (kk % 4) * 32) >> 4;
                                 mma_ss(tmem, a + off16, b + off16, idesc_qk, kk > 0);
                             }

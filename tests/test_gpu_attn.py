@@ -36,6 +36,11 @@ def run_attn(basp, w, causal=True, scale=0.0, seed=0, with_lse=True):
     ("one_tile", synth.Workload("one_tile", N=1, B=1, S=128, Hq=1, Hkv=1, D=128)),
     ("ragged_tiles", synth.Workload("ragged", N=2, B=2, S=640, Hq=2, Hkv=1, D=64)),
     ("ulysses", synth.Workload("ulysses", N=4, B=2, S=512, Hq=8, Hkv=4, D=128, G=1)),
+    ("head_dim_96", synth.Workload("d96", N=4, B=2, S=640, Hq=8, Hkv=4, D=96)),       # hidden 3072 / 32 heads
+    ("head_dim_96_ragged", synth.Workload("d96r", N=2, B=2, S=333, Hq=4, Hkv=2, D=96)),
+    ("head_dim_80", synth.shrink(synth.WORKLOADS["t2_qwen25_3b"], 256)),                # hidden 2560 / 32 heads
+    ("head_dim_48", synth.Workload("d48", N=2, B=2, S=384, Hq=4, Hkv=4, D=48)),
+    ("head_dim_112", synth.Workload("d112", N=2, B=1, S=512, Hq=4, Hkv=2, D=112)),
 ])
 def test_attn_fwd_matches_oracle(basp, name, w):
     got, ref, lse, ref_lse = run_attn(basp, w)

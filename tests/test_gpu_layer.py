@@ -32,6 +32,7 @@ def gpu_layer(basp, w, Xq, Xk, Xv, op, fused):
     synth.shrink(synth.WORKLOADS["sweep_b1"], 128),
     synth.shrink(synth.WORKLOADS["sweep_b8"], 256),
     synth.shrink(synth.WORKLOADS["qwen25_7b_64k"], 128),
+    synth.Workload("head_dim_96", N=4, B=2, S=512, Hq=8, Hkv=4, D=96),
 ], ids=lambda w: w.name)
 def test_layer_matches_oracle(basp, w, fused):
     Xq, Xk, Xv, op = oracle_inputs(w)

@@ -77,6 +77,6 @@ def test_null_and_alignment_checks_need_no_gpu(basp):
         == basp.BASP_ERR_WORKSPACE
     pl2 = basp.basp_plan_create(4, 2, 1000, 8, 8, 64)    # T = 500 is not a multiple of 128: tiles would straddle ranks
     assert L.basp_layer_fwd_fused(pl2.handle, good, good, good, good2, None, 0.0, None) == basp.BASP_ERR_UNSUPPORTED
-    pl3 = basp.basp_plan_create(4, 2, 1024, 8, 8, 32)    # head dim the kernels do not implement
+    pl3 = basp.basp_plan_create(4, 2, 1024, 8, 8, 40)    # head dim the kernels do not implement (not a multiple of 16)
     assert L.basp_attn_fwd(pl3.handle, good, good, good, good2, None, 0.0, None) == basp.BASP_ERR_UNSUPPORTED
     assert basp.lib.basp_strerror(-7).decode().startswith("a bounded wait")
