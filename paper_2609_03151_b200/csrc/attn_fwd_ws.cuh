@@ -409,9 +409,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                         const uint64_t a = desc_k | (uint64_t)(q_addr16 + t * (kTileBytes >> 4));
                         const uint64_t b = desc_k | (uint64_t)(kv_addr16 + slot * (kTileBytes >> 4));
                         if (lane == 0) {
+                            // all D/16 steps even when the head dimension is smaller: the padding columns are zero, and a
+                            // per-MMA test in this loop costs more (12 % of the kernel) than the two or three extra MMAs
 #pragma unroll
                             for (int kk = 0; kk < D / 16; ++kk) {
-                                if (kk * 16 >= p.Dg) break;   // zero padding contributes nothing to Q.K^T
                                 const uint32_t off16 = ((kk / 4) * 16384 + (kk % 4) * 32) >> 4;
                                 mma_ss(tmem, a + off16, b + off16, idesc_qk, kk > 0);
                             }
