@@ -77,7 +77,8 @@ typedef struct basp_plan_info {
     int q_heads_per_rank;  /* Hq / K                                                      */
     int kv_heads_per_rank; /* Hkv / K                                                     */
     size_t q_shard_elems;  /* elements of one rank's Q (or O) shard, either layout        */
-    size_t kv_shard_elems; /* elements of one rank's K (or V) shard, either layout        */
+    size_t kv_shard_elems; /* elements of one rank's K (or V) shard (sequence-sharded;    */
+                           /* head-sharded too unless KV heads are replicated, see below)  */
     size_t lse_shard_elems;/* fp32 elements of one rank's LSE                             */
 } basp_plan_info;
 
@@ -95,8 +96,13 @@ typedef struct basp_rank_info {
  * as in the workload-equivalence paragraph of Section IV-C.
  * Errors: BASP_ERR_NULL; BASP_ERR_INVALID for N mod G != 0, B mod G != 0, B > N in BASP
  * mode (the paper's data-parallel fallback is not provided), S mod K != 0, Hq mod Hkv != 0,
- * Hq mod K != 0, Hkv mod K != 0; BASP_ERR_UNSUPPORTED for dtype != bf16, N > BASP_MAX_RANKS
- * or a head slice whose row ((H/K)*D*2 bytes) is not a multiple of 16 bytes.
+ * Hq mod K != 0, or Hkv and K with neither Hkv mod K = 0 nor K mod Hkv = 0; BASP_ERR_UNSUPPORTED for
+ * dtype != bf16, N > BASP_MAX_RANKS or a head slice whose row ((H/K)*D*2 bytes) is not a multiple of 16 bytes.
+ * A group with MORE ranks than KV heads (K mod Hkv = 0, K > Hkv; the paper does not treat grouped-query attention)
+ * replicates: KV head h is delivered to the K/Hkv consecutive local ranks whose query heads read it, so every rank
+ * holds one KV head (kv_heads_per_rank = 1, kv_head_begin = local_rank / (K/Hkv)); its head-sharded K or V shard is
+ * [Bl][S][1][D], larger than the sequence-sharded one.  Forward only: basp_reshard_h2s of such a tensor and the
+ * backward calls return BASP_ERR_UNSUPPORTED (the gradients of the copies would have to be added up).
  * On success *out owns a host object; release it with basp_plan_destroy. */
 int basp_plan_create(const basp_config *cfg, basp_plan **out);
 int basp_plan_destroy(basp_plan *plan);

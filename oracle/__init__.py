@@ -127,6 +127,23 @@ def s2h(seq: np.ndarray, pl: Plan) -> np.ndarray:
     return out
 
 
+def s2h_replicated(seq: np.ndarray, pl: Plan) -> np.ndarray:
+    """First all-to-all for a K/V tensor with FEWER heads than the group has ranks (K mod H = 0): local rank m needs
+    the KV head that its query heads read, head m // (K/H), over the whole sequence, so each head is delivered to K/H
+    consecutive local ranks.  seq [N,Bl,T,H,D] -> [N,Bl,S,1,D].  (The paper does not treat grouped-query attention;
+    this is the head mapping h -> h / (Hq/Hkv) applied to the contiguous query-head blocks of Section IV-C.)"""
+    seq = np.ascontiguousarray(seq)
+    N, Bl, T, H, D = seq.shape
+    assert (N, Bl, T) == (pl.N, pl.Bl, pl.T) and pl.K % H == 0 and H < pl.K
+    rep = pl.K // H
+    out = np.empty((N, Bl, pl.S, 1, D), dtype=seq.dtype)
+    for g in range(pl.G):
+        for m in range(pl.K):                      # destination local rank
+            for src in range(pl.K):                # source local rank = chunk of the sequence
+                out[g * pl.K + m, :, src * T:(src + 1) * T, 0, :] = seq[g * pl.K + src, :, :, m // rep, :]
+    return out
+
+
 def h2s(head: np.ndarray, pl: Plan) -> np.ndarray:
     """Group-local all-to-all, head-sharded -> sequence-sharded (the reverse one)."""
     head = np.ascontiguousarray(head)
@@ -247,7 +264,8 @@ def layer_fwd(Xq: np.ndarray, Xk: np.ndarray, Xv: np.ndarray, pl: Plan,
     Xq [B,S,Hq,D], Xk,Xv [B,S,Hkv,D] uint16.  Returns a dict with every intermediate
     (seq shards, head shards, per-rank O/LSE in fp64) and the global O [B,S,Hq,D]."""
     qs, ks, vs = partition(Xq, pl), partition(Xk, pl), partition(Xv, pl)
-    qh, kh, vh = s2h(qs, pl), s2h(ks, pl), s2h(vs, pl)
+    kv_s2h = s2h if Xk.shape[2] % pl.K == 0 else s2h_replicated
+    qh, kh, vh = s2h(qs, pl), kv_s2h(ks, pl), kv_s2h(vs, pl)
     N = pl.N
     oh = np.empty(qh.shape, dtype=np.float64)
     lse = np.empty((N, pl.Bl, qh.shape[3], pl.S), dtype=np.float64)

@@ -65,7 +65,8 @@ void oracle_group_ranks(int K, int group, int *ranks_out) {
 
 /* Algorithm 2 for one rank: group = floor(r / K), local = r mod K, the
  * sequences [group*Bl, (group+1)*Bl) and the tokens [local*T, (local+1)*T);
- * head blocks are the contiguous split of H heads into K parts.
+ * head blocks are the contiguous split of H heads into K parts (KV heads: see below
+ * for a group with more ranks than KV heads).
  * out = {group, local, seq_begin, seq_end, token_begin, token_end,
  *        q_head_begin, q_head_end, kv_head_begin, kv_head_end}. */
 void oracle_rank_info(int K, int Bl, int T, int Hq, int Hkv, int r, int out[10]) {
@@ -78,8 +79,16 @@ void oracle_rank_info(int K, int Bl, int T, int Hq, int Hkv, int r, int out[10])
     out[5] = (l + 1) * T;
     out[6] = l * (Hq / K);
     out[7] = (l + 1) * (Hq / K);
-    out[8] = l * (Hkv / K);
-    out[9] = (l + 1) * (Hkv / K);
+    if (Hkv % K == 0) {
+        out[8] = l * (Hkv / K);
+        out[9] = (l + 1) * (Hkv / K);
+    } else {
+        /* more ranks in the group than KV heads (the paper does not treat grouped-query
+         * attention): query head h reads KV head h / (Hq/Hkv), so the K/Hkv consecutive
+         * local ranks whose query heads share a KV head each hold that one head. */
+        out[8] = l / (K / Hkv);
+        out[9] = out[8] + 1;
+    }
 }
 
 /* ------------------------------------------------------------------------- */

@@ -581,7 +581,7 @@ extern "C" int basp_attn_bwd(const basp_plan *pl, const void *const *q_head, con
     if (!pl || !q_head || !k_head || !v_head || !o_head || !do_head || !lse_shards || !dq_head || !dk_head ||
         !dv_head || !workspace)
         return BASP_ERR_NULL;
-    if (pl->D != 128 || pl->S % kT != 0) return BASP_ERR_UNSUPPORTED;
+    if (pl->D != 128 || pl->S % kT != 0 || pl->kv_rep != 1) return BASP_ERR_UNSUPPORTED;
     if (!aligned16(workspace)) return BASP_ERR_ALIGN;
     if (workspace_bytes < basp_attn_bwd_workspace_bytes(pl)) return BASP_ERR_WORKSPACE;
     for (int r = 0; r < pl->N; ++r) {

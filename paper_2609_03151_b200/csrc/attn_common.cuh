@@ -17,7 +17,8 @@ struct AttnParams {
     CUtensorMap q[R], k[R], v[R];
     __nv_bfloat16 *o[R];
     float *lse[R];
-    int n_ranks, K, Bl, S, T, Hq_l, Hkv_l, q_per_kv;
+    int n_ranks, K, Bl, S, T, Hq_l, Hkv_l, q_per_kv;   // q_per_kv: query heads per KV head on a rank
+    int kv_rep;             // local ranks sharing one KV head (sequence-sharded K/V: head index = local rank / kv_rep)
     int o_heads;            // heads in one row of the O destination (Hq_l, or Hq when fused)
     int Dg;                 // head dimension in memory, a multiple of 16 up to the kernel's width (64 or 128): the tile
                             // loads zero-fill the columns past it, the products skip them, the epilogue does not store them
@@ -36,14 +37,15 @@ struct TileCoord {
 // Where the 128-token tile starting at sequence position s0 of (rank r, sequence bl, local
 // head h) is found.  `heads_l` is the number of local heads of that tensor.
 template <int R>
-__device__ __forceinline__ TileCoord locate(const AttnParams<R> &p, int r, int bl, int s0, int h, int heads_l) {
+__device__ __forceinline__ TileCoord locate(const AttnParams<R> &p, int r, int bl, int s0, int h, int heads_l,
+                                            int rep = 1) {
     TileCoord c;
     if (p.fused) {
         const int g = r / p.K, l = r - g * p.K;
         const int owner = s0 / p.T;
         c.rank = g * p.K + owner;
         c.row = bl * p.T + (s0 - owner * p.T);
-        c.head = l * heads_l + h;
+        c.head = rep > 1 ? l / rep : l * heads_l + h;
     } else {
         c.rank = r;
         c.row = bl * p.S + s0;

@@ -51,11 +51,12 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
         prm.lse[r] = lse ? lse[r] : nullptr;
     }
     prm.n_ranks = pl->N; prm.K = pl->K; prm.Bl = pl->Bl; prm.S = pl->S; prm.T = pl->T;
-    prm.Hq_l = pl->Hq_l; prm.Hkv_l = pl->Hkv_l; prm.q_per_kv = pl->Hq / pl->Hkv;
+    prm.Hq_l = pl->Hq_l; prm.Hkv_l = pl->Hkv_l; prm.q_per_kv = pl->Hq_l / pl->Hkv_l;
+    prm.kv_rep = pl->kv_rep;
     prm.o_heads = hq;
     prm.Dg = pl->D;
     {
-        const int q_per_kv = pl->Hq / pl->Hkv;
+        const int q_per_kv = pl->Hq_l / pl->Hkv_l;
         prm.r_begin = range[0]; prm.r_count = range[1]; prm.qb_begin = range[2]; prm.qb_count = range[3];
         int band = BASP_BAND_TARGET / q_per_kv < 1 ? 1 : (BASP_BAND_TARGET / q_per_kv > 16 ? 16 : BASP_BAND_TARGET / q_per_kv);
         while (prm.qb_count % band != 0) --band;

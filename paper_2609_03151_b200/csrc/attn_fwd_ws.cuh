@@ -363,7 +363,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                             tma_load_3d(sQ + t * kTileBytes + s * 16384, &p.q[c.rank], &sh.q_full, s * 64, c.head, c.row);
                 }
                 for (int j = 0; j < item.n_max; ++j) {
-                    const TileCoord c = locate(p, item.r, item.bl, j * kTile, item.hkv, p.Hkv_l);
+                    const TileCoord c = locate(p, item.r, item.bl, j * kTile, item.hkv, p.Hkv_l, p.kv_rep);
 #pragma unroll
                     for (int x = 0; x < 2; ++x, ++kv_it) {
                         const uint32_t slot = kv_it % kStages, ph = (kv_it / kStages) & 1;

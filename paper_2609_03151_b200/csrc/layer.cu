@@ -13,11 +13,13 @@ int basp_attn_dispatch_range(const basp_plan *pl, const void *const *q, const vo
 namespace {
 size_t q_shard_bytes(const basp_plan *p) { return (size_t)p->Bl * p->T * p->Hq * p->D * 2; }
 size_t kv_shard_bytes(const basp_plan *p) { return (size_t)p->Bl * p->T * p->Hkv * p->D * 2; }
+// head-sharded K or V of one rank: the same bytes unless KV heads are replicated inside the group
+size_t kv_head_bytes(const basp_plan *p) { return (size_t)p->Bl * p->S * p->Hkv_l * p->D * 2; }
 }  // namespace
 
 extern "C" size_t basp_workspace_bytes(const basp_plan *p) {
     if (!p) return 0;
-    return (size_t)p->N * (2 * q_shard_bytes(p) + 2 * kv_shard_bytes(p));   // head-sharded Q, K, V, O
+    return (size_t)p->N * (2 * q_shard_bytes(p) + 2 * kv_head_bytes(p));   // head-sharded Q, K, V, O
 }
 
 extern "C" size_t basp_host_arena_bytes(const basp_plan *p) { return basp_workspace_bytes(p); }
@@ -30,7 +32,7 @@ extern "C" int basp_layer_fwd(const basp_plan *p, const void *const *q_seq, cons
     if (workspace_bytes < basp_workspace_bytes(p)) return BASP_ERR_WORKSPACE;
     char *w = (char *)workspace;
     void *qh[BASP_MAX_RANKS], *kh[BASP_MAX_RANKS], *vh[BASP_MAX_RANKS], *oh[BASP_MAX_RANKS];
-    const size_t qb = q_shard_bytes(p), kb = kv_shard_bytes(p);
+    const size_t qb = q_shard_bytes(p), kb = kv_head_bytes(p);
     for (int r = 0; r < p->N; ++r) {
         qh[r] = w + (size_t)r * qb;
         kh[r] = w + (size_t)p->N * qb + (size_t)r * kb;
@@ -48,7 +50,7 @@ extern "C" int basp_layer_workspace_shards(const basp_plan *p, void *workspace, 
                                            void **v_head, void **o_head) {
     if (!p || !workspace || !q_head || !k_head || !v_head || !o_head) return BASP_ERR_NULL;
     char *w = (char *)workspace;
-    const size_t qb = q_shard_bytes(p), kb = kv_shard_bytes(p);
+    const size_t qb = q_shard_bytes(p), kb = kv_head_bytes(p);
     for (int r = 0; r < p->N; ++r) {
         q_head[r] = w + (size_t)r * qb;
         k_head[r] = w + (size_t)p->N * qb + (size_t)r * kb;

@@ -17,16 +17,20 @@ extern "C" int basp_plan_create(const basp_config *cfg, basp_plan **out) {
     if (N % G != 0 || B % G != 0) return BASP_ERR_INVALID;      // Algorithm 1: assert N mod B = 0
     const int K = N / G;                                         // Algorithm 1: K = N / B
     if (S % K != 0) return BASP_ERR_INVALID;                     // Algorithm 2: chunk = L / K
-    if (Hq % Hkv != 0 || Hq % K != 0 || Hkv % K != 0) return BASP_ERR_INVALID;
+    // Each rank takes Hq/K query heads and their KV heads.  A group with more ranks than KV heads replicates: KV head
+    // h goes to the K/Hkv consecutive local ranks whose query heads read it (one KV head per rank).
+    if (Hq % Hkv != 0 || Hq % K != 0) return BASP_ERR_INVALID;
+    if (Hkv % K != 0 && K % Hkv != 0) return BASP_ERR_INVALID;
+    const int kv_rep = Hkv % K == 0 ? 1 : K / Hkv, Hkv_l = Hkv % K == 0 ? Hkv / K : 1;
     if (cfg->dtype != BASP_DTYPE_BF16 || N > BASP_MAX_RANKS) return BASP_ERR_UNSUPPORTED;
-    if (((Hkv / K) * D * 2) % 16 != 0 || ((Hq / K) * D * 2) % 16 != 0) return BASP_ERR_UNSUPPORTED;
+    if ((Hkv_l * D * 2) % 16 != 0 || ((Hq / K) * D * 2) % 16 != 0) return BASP_ERR_UNSUPPORTED;
     if (cfg->causal != 0 && cfg->causal != 1) return BASP_ERR_INVALID;
 
     basp_plan *p = new (std::nothrow) basp_plan;
     if (!p) return BASP_ERR_INVALID;
     p->cfg = *cfg;
     p->N = N; p->B = B; p->G = G; p->K = K; p->Bl = B / G; p->S = S; p->T = S / K;
-    p->Hq = Hq; p->Hkv = Hkv; p->D = D; p->Hq_l = Hq / K; p->Hkv_l = Hkv / K;
+    p->Hq = Hq; p->Hkv = Hkv; p->D = D; p->Hq_l = Hq / K; p->Hkv_l = Hkv_l; p->kv_rep = kv_rep;
     p->causal = cfg->causal;
     *out = p;
     return BASP_OK;
@@ -65,8 +69,8 @@ extern "C" int basp_plan_get_rank(const basp_plan *p, int r, basp_rank_info *inf
     info->token_end = (l + 1) * p->T;
     info->q_head_begin = l * p->Hq_l;
     info->q_head_end = (l + 1) * p->Hq_l;
-    info->kv_head_begin = l * p->Hkv_l;
-    info->kv_head_end = (l + 1) * p->Hkv_l;
+    info->kv_head_begin = p->kv_rep > 1 ? l / p->kv_rep : l * p->Hkv_l;
+    info->kv_head_end = info->kv_head_begin + p->Hkv_l;
     return BASP_OK;
 }
 

@@ -7,6 +7,7 @@ struct basp_plan {
     int N, B, G, K, Bl, S, T;
     int Hq, Hkv, D;
     int Hq_l, Hkv_l;   // heads per rank after the first all-to-all
+    int kv_rep;        // ranks of a group that hold the same KV head (1 unless the group has more ranks than KV heads)
     int causal;
 };
 

@@ -24,7 +24,8 @@ struct ReshardTensor {
     const char *seq[BASP_MAX_RANKS];
     const char *head[BASP_MAX_RANKS];
     uint32_t row_v;            // vectors per token row on the sequence-sharded side (K runs)
-    uint32_t run_v;            // vectors per run = (H/K)*D*2/16
+    uint32_t run_v;            // vectors per run = (H/K)*D*2/16 (one head when replicated)
+    uint32_t rep;              // head-side ranks that receive each run (1; K/H when a group has more ranks than heads)
     uint32_t shard_v;          // vectors per rank shard
     uint32_t chunks_per_shard;
     uint32_t chunk_begin;      // first CTA index of this tensor
@@ -66,7 +67,8 @@ __global__ void __launch_bounds__(kThreads) reshard_kernel(const __grid_constant
     const uint32_t v0 = chunk * kChunkV + threadIdx.x;
 
     const uint4 *seq = reinterpret_cast<const uint4 *>(t.seq[r]);
-    const uint4 *hp[kUnroll];   // address on the head-sharded side of each vector
+    const uint4 *hp[kUnroll];   // address on the head-sharded side of each vector (of its first copy when replicated)
+    uint32_t hrank[kUnroll], hoff[kUnroll];
 #pragma unroll
     for (int i = 0; i < kUnroll; ++i) {
         const uint32_t v = v0 + i * kThreads;
@@ -78,7 +80,9 @@ __global__ void __launch_bounds__(kThreads) reshard_kernel(const __grid_constant
         const uint32_t bl = fdiv(tok, p.div_T);
         const uint32_t tt = tok - bl * p.T;
         const uint32_t hv = (bl * p.S + l * p.T + tt) * t.run_v + j;
-        hp[i] = reinterpret_cast<const uint4 *>(t.head[g * p.K + m]) + hv;
+        hrank[i] = g * p.K + m * t.rep;
+        hoff[i] = hv;
+        hp[i] = reinterpret_cast<const uint4 *>(t.head[hrank[i]]) + hv;
     }
     uint4 data[kUnroll];
 #pragma unroll
@@ -91,6 +95,15 @@ __global__ void __launch_bounds__(kThreads) reshard_kernel(const __grid_constant
         const uint32_t v = v0 + i * kThreads;
         if (v < t.shard_v) st_stream(const_cast<uint4 *>(kToHead ? hp[i] : seq + v), data[i]);
     }
+    if (kToHead && t.rep > 1) {         // the other local ranks that read this KV head get the same run
+        for (uint32_t c = 1; c < t.rep; ++c)
+#pragma unroll
+            for (int i = 0; i < kUnroll; ++i) {
+                const uint32_t v = v0 + i * kThreads;
+                if (v < t.shard_v)
+                    st_stream(const_cast<uint4 *>(reinterpret_cast<const uint4 *>(t.head[hrank[i] + c]) + hoff[i]), data[i]);
+            }
+    }
 }
 
 struct TensorArg {
@@ -102,11 +115,16 @@ struct TensorArg {
 int fill_tensor(const basp_plan *p, const TensorArg &a, bool to_head, int r_begin, int r_count, ReshardTensor *t,
                 uint32_t *chunk_cursor) {
     if (!a.seq || !a.head) return BASP_ERR_NULL;
-    if (a.n_heads <= 0 || a.n_heads % p->K != 0) return BASP_ERR_INVALID;
-    const size_t run_bytes = (size_t)(a.n_heads / p->K) * p->D * 2;
+    if (a.n_heads <= 0) return BASP_ERR_INVALID;
+    // fewer heads than ranks in a group (KV heads under GQA): every head goes to K/H consecutive local ranks
+    const int rep = a.n_heads % p->K == 0 ? 1 : (p->K % a.n_heads == 0 ? p->K / a.n_heads : 0);
+    if (rep == 0) return BASP_ERR_INVALID;
+    if (rep > 1 && !to_head) return BASP_ERR_UNSUPPORTED;       // the way back would have to add the copies up
+    const size_t run_bytes = (rep > 1 ? (size_t)1 : (size_t)(a.n_heads / p->K)) * p->D * 2;
     if (run_bytes % 16 != 0) return BASP_ERR_UNSUPPORTED;
-    const size_t shard_bytes = (size_t)p->Bl * p->T * a.n_heads * p->D * 2;
-    if (shard_bytes / 16 >= (1ull << 31)) return BASP_ERR_UNSUPPORTED;
+    const size_t shard_bytes = (size_t)p->Bl * p->T * a.n_heads * p->D * 2;                 // sequence side
+    const size_t head_bytes = rep > 1 ? (size_t)p->Bl * p->S * p->D * 2 : shard_bytes;          // head side
+    if (head_bytes / 16 >= (1ull << 31)) return BASP_ERR_UNSUPPORTED;
     // The launch walks the sequence-side shards of ranks [r_begin, r_begin + r_count) and touches the head-side
     // shards of every member of their groups; the other entries are not read (they may be NULL).
     const int g_begin = r_begin / p->K * p->K, g_end = (r_begin + r_count + p->K - 1) / p->K * p->K;
@@ -121,10 +139,11 @@ int fill_tensor(const basp_plan *p, const TensorArg &a, bool to_head, int r_begi
     for (int i = r_begin; i < r_begin + r_count; ++i)
         for (int j = g_begin; j < g_end; ++j) {
             const char *s = t->seq[i], *d = t->head[j];
-            if (s < d + shard_bytes && d < s + shard_bytes) return BASP_ERR_ALIAS;
+            if (s < d + head_bytes && d < s + shard_bytes) return BASP_ERR_ALIAS;
         }
+    t->rep = (uint32_t)rep;
     t->run_v = (uint32_t)(run_bytes / 16);
-    t->row_v = t->run_v * p->K;
+    t->row_v = t->run_v * (rep > 1 ? (uint32_t)a.n_heads : (uint32_t)p->K);
     t->shard_v = (uint32_t)(shard_bytes / 16);
     t->chunks_per_shard = (t->shard_v + kChunkV - 1) / kChunkV;
     t->chunk_begin = *chunk_cursor;

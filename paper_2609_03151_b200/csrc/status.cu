@@ -87,7 +87,7 @@ extern "C" int basp_selftest_wait_timeout(unsigned int limit_us, void *stream) {
 extern "C" const char *basp_strerror(int code) {
     switch (code) {
         case BASP_OK: return "ok";
-        case BASP_ERR_INVALID: return "invalid plan or argument (N mod G, B > N, S mod K, head split)";
+        case BASP_ERR_INVALID: return "invalid plan or argument (N mod G, B > N, S mod K, head split, rank range)";
         case BASP_ERR_UNSUPPORTED: return "valid but not implemented by the kernels";
         case BASP_ERR_NULL: return "null pointer";
         case BASP_ERR_ALIGN: return "device pointer not 16-byte aligned";

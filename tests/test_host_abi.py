@@ -33,6 +33,18 @@ def test_plan_matches_oracle(basp, N, B, G):
         assert basp.basp_plan_get_rank(pl, r) == op.rank_info(r, Hq, Hkv)
 
 
+@pytest.mark.parametrize("N,B,Hq,Hkv", [(8, 2, 32, 2), (8, 1, 32, 4), (4, 1, 8, 1)])
+def test_plan_with_more_ranks_than_kv_heads(basp, N, B, Hq, Hkv):
+    """A group with more ranks than KV heads: one (replicated) KV head per rank, as the oracle reads it."""
+    S, D = 2048, 128
+    pl = basp.basp_plan_create(N, B, S, Hq, Hkv, D)
+    op = oracle.plan(N, B, S)
+    assert pl.K > Hkv and pl.info.kv_heads_per_rank == 1 and pl.info.q_heads_per_rank == Hq // pl.K
+    assert pl.info.kv_shard_elems == B * S // N * Hkv * D       # the sequence-sharded side is unchanged
+    for r in range(N):
+        assert basp.basp_plan_get_rank(pl, r) == op.rank_info(r, Hq, Hkv)
+
+
 def test_paper_example_four_gpus_batch_two(basp):
     pl = basp.basp_plan_create(4, 2, 1024, 8, 8, 64)
     assert pl.K == 2 and [basp.basp_plan_group_ranks(pl, g) for g in range(2)] == [[0, 1], [2, 3]]
@@ -43,7 +55,7 @@ def test_paper_example_four_gpus_batch_two(basp):
     (dict(n_ranks=4, micro_batch=8), -1),                 # B > N
     (dict(seq_len=1022), -1),                             # S mod K != 0
     (dict(n_q_heads=30), -1),                             # Hq mod Hkv
-    (dict(n_kv_heads=2), -1),                             # Hkv mod K (K = 4)
+    (dict(n_ranks=6, micro_batch=1, seq_len=1536, n_q_heads=24, n_kv_heads=4), -1),   # K = 6: neither Hkv mod K nor K mod Hkv
     (dict(num_groups=3), -1),
     (dict(dtype=1), -2),
     (dict(n_ranks=64, micro_batch=64), -2),               # more than BASP_MAX_RANKS
