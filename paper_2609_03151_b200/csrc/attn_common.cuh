@@ -28,6 +28,9 @@ struct AttnParams {
     int fused, causal, has_lse;
     float scale_log2;       // softmax scale * log2(e)
     int *status;
+    // divisors of the item decoding, prepared on the host (a division by a runtime value is some 25 instructions, and
+    // the decoding is inlined into every role: instruction fetch matters in this kernel)
+    FastDiv div_per_band, div_per_stream, div_q_per_kv, div_hkv_l, div_bl;
 };
 
 struct TileCoord {

@@ -61,6 +61,11 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
         int band = BASP_BAND_TARGET / q_per_kv < 1 ? 1 : (BASP_BAND_TARGET / q_per_kv > 16 ? 16 : BASP_BAND_TARGET / q_per_kv);
         while (prm.qb_count % band != 0) --band;
         prm.qb_band = band;
+        prm.div_per_band = make_fastdiv((uint32_t)(range[1] * pl->Bl * pl->Hq_l * band));
+        prm.div_per_stream = make_fastdiv((uint32_t)(band * q_per_kv));
+        prm.div_q_per_kv = make_fastdiv((uint32_t)q_per_kv);
+        prm.div_hkv_l = make_fastdiv((uint32_t)pl->Hkv_l);
+        prm.div_bl = make_fastdiv((uint32_t)pl->Bl);
     }
     prm.fused = fused; prm.causal = pl->causal; prm.has_lse = lse != nullptr;
     prm.scale_log2 = (scale == 0.f ? 1.f / sqrtf((float)pl->D) : scale) * 1.4426950408889634f;

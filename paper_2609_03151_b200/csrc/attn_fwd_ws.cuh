@@ -54,19 +54,18 @@ __device__ __forceinline__ bool ws_get_item(const AttnParams<R> &p, int round, W
     // Order: bands of `qb_band` consecutive query blocks, longest first; inside a band the items of
     // one KV stream (rank, sequence, KV head) are adjacent -- qb_band blocks x q_per_kv query heads --
     // so that the CTAs running side by side read the same K/V tiles through L2.
-    const int per_band = per_qb * p.qb_band;
-    const int band = i / per_band;
-    int rem = i - band * per_band;
-    const int per_stream = p.qb_band * p.q_per_kv;
-    const int stream = rem / per_stream;
-    rem -= stream * per_stream;
-    const int qb_in_band = rem / p.q_per_kv;
+    const int band = (int)fdiv((uint32_t)i, p.div_per_band);
+    int rem = i - band * (int)p.div_per_band.d;
+    const int stream = (int)fdiv((uint32_t)rem, p.div_per_stream);
+    rem -= stream * (int)p.div_per_stream.d;
+    const int qb_in_band = (int)fdiv((uint32_t)rem, p.div_q_per_kv);
     it.qb = p.qb_begin + p.qb_count - 1 - (band * p.qb_band + qb_in_band);
-    it.hkv = stream % p.Hkv_l;
+    const int sb = (int)fdiv((uint32_t)stream, p.div_hkv_l);
+    it.hkv = stream - sb * p.Hkv_l;
     it.h = it.hkv * p.q_per_kv + (rem - qb_in_band * p.q_per_kv);
-    const int sb = stream / p.Hkv_l;
-    it.bl = sb % p.Bl;
-    it.r = p.r_begin + sb / p.Bl;
+    const int rr = (int)fdiv((uint32_t)sb, p.div_bl);
+    it.bl = sb - rr * p.Bl;
+    it.r = p.r_begin + rr;
     const int qt0 = 2 * it.qb, qt1 = qt0 + 1;
     const bool has1 = qt1 < n_qt;
     it.n[0] = p.causal ? qt0 + 1 : n_qt;
@@ -273,7 +272,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
             const int s_pos = (2 * item.qb + t) * kTile + row;
             if (p.has_lse && s_pos < p.S) {
                 p.lse[item.r][((size_t)item.bl * p.Hq_l + item.h) * p.S + s_pos] =
-                    m_ref * 0.6931471805599453f + logf(l_run);
+                    m_ref * 0.6931471805599453f + __logf(l_run);
             }
         }
     } else if (warp < 12) {
@@ -298,7 +297,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                     if (j > 0 && !__all_sync(0xffffffffu, alpha == 1.f)) {
                         tc_fence_after();
                         const uint32_t O_t = tmem + 256 + 128 * t + lane_addr;
-#pragma unroll
+#pragma unroll 1                 // rare and not time-critical: kept small
                         for (int c = 0; c < kOCols / 32; ++c) {
                             uint32_t rr[32];
                             tmem_ld_x32(O_t + c * 32, rr);

@@ -54,7 +54,7 @@ constexpr uint64_t kWaitLimitNs = 2000ull * 1000ull * 1000ull;   // 2 s
 
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
                                           uint32_t sleep_ns = 0, uint64_t limit_ns = kWaitLimitNs) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (__builtin_expect(mbar_try_wait(bar, parity), 1)) return true;    // the spinning part is laid out away from the hot code
     const uint64_t t0 = globaltimer_ns();
     uint32_t spins = 0;
     while (true) {
