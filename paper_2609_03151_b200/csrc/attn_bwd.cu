@@ -93,7 +93,7 @@ __device__ __forceinline__ void bwd_report(int *status, int code, int role, int 
 #ifdef BASP_PHASE_TIMING
 __device__ long long g_bwd_phase[32];
 #define BPH_T(var) const long long var = clock64()
-#define BPH_ADD(slot, a, b) do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (warp == 0 || warp == kBwdMmaWarp || warp == kBwdDrainWarp0)) g_bwd_phase[slot] += (b) - (a); } while (0)
+#define BPH_ADD(slot, a, b) do { bacc[(slot) & 7] += (b) - (a); } while (0)
 #else
 #define BPH_T(var)
 #define BPH_ADD(slot, a, b)
@@ -123,6 +123,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     BwdBars *bars = reinterpret_cast<BwdBars *>(s_delta + 2 * kT);
 
     const int tid = threadIdx.x, warp = __shfl_sync(0xffffffffu, tid >> 5, 0), lane = tid & 31;
+#ifdef BASP_PHASE_TIMING
+    long long bacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#endif
 
     if (tid == 0) {
         mbar_init(&bars->kv_full, 1); mbar_init(&bars->kv_empty, 1);
@@ -167,6 +170,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     const int buf = it_g & 1;
                     BPH_T(t0);
                     BWD_WAIT(&bars->stats_full[buf], (it_g >> 1) & 1, 10, m);   // LSE and Delta of the query tile (producer warp)
+                    BPH_T(t0a);
+                    BPH_ADD(7, t0, t0a);
                     BWD_WAIT(&bars->s_full, it_g & 1, 11, m);
                     tc_fence_after();
                     BPH_T(t1);
@@ -214,7 +219,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     BPH_T(t4);
                     BPH_T(t5);
                     BPH_T(t6);
-                    BPH_ADD(0, t0, t1); BPH_ADD(1, t1, t2); BPH_ADD(2, t2, t3); BPH_ADD(3, t3, t4);
+                    BPH_ADD(0, t0a, t1); BPH_ADD(1, t1, t2); BPH_ADD(2, t2, t3); BPH_ADD(3, t3, t4);
                     BPH_ADD(4, t4, t5); BPH_ADD(5, t5, t6); BPH_ADD(6, t0, t0 + 1);
                 }
             }
@@ -446,6 +451,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     }
 
 bwd_done:
+#ifdef BASP_PHASE_TIMING
+    if (blockIdx.x == 5 && (threadIdx.x & 31) == 0 && (warp == 0 || warp == kBwdMmaWarp || warp == kBwdDrainWarp0)) {
+        const int base_ = warp == 0 ? 0 : (warp == kBwdMmaWarp ? 8 : 16);
+        for (int i_ = 0; i_ < 8; ++i_) g_bwd_phase[base_ + i_] += bacc[i_];
+    }
+#endif
     tc_fence_before();
     __syncthreads();
     if (bars->abort_flag) {
