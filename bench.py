@@ -37,7 +37,7 @@ DEFAULT_WORKLOAD = "llama3_8b_32k"          # BASELINE config 2: N=8, b=2, S=327
 # DRAM bytes (read + write) of one attention launch from an ncu capture, per workload; None = not captured.
 NCU_TRAFFIC_BYTES = {
     # profiles/attn_fwd_ws_traffic_llama3_8b_32k.md: dram__bytes_read.sum + dram__bytes_write.sum of one launch
-    "llama3_8b_32k": 2970402560 + 529428992,
+    "llama3_8b_32k": 3033940992 + 539852800,
 }
 
 
