@@ -101,8 +101,9 @@ typedef struct basp_rank_info {
  * A group with MORE ranks than KV heads (K mod Hkv = 0, K > Hkv; the paper does not treat grouped-query attention)
  * replicates: KV head h is delivered to the K/Hkv consecutive local ranks whose query heads read it, so every rank
  * holds one KV head (kv_heads_per_rank = 1, kv_head_begin = local_rank / (K/Hkv)); its head-sharded K or V shard is
- * [Bl][S][1][D], larger than the sequence-sharded one.  Forward only: basp_reshard_h2s of such a tensor and the
- * backward calls return BASP_ERR_UNSUPPORTED (the gradients of the copies would have to be added up).
+ * [Bl][S][1][D], larger than the sequence-sharded one.  On the way back such a tensor carries gradients:
+ * basp_reshard_h2s (and basp_reshard_grads_h2s for dK, dV) ADDS the K/Hkv copies of a head (fp32 sum, one rounding),
+ * which is what the backward pass needs; basp_reshard_h2s is therefore not the inverse of basp_reshard_s2h for it.
  * On success *out owns a host object; release it with basp_plan_destroy. */
 int basp_plan_create(const basp_config *cfg, basp_plan **out);
 int basp_plan_destroy(basp_plan *plan);

@@ -144,6 +144,22 @@ def s2h_replicated(seq: np.ndarray, pl: Plan) -> np.ndarray:
     return out
 
 
+def h2s_sum_replicated(head: np.ndarray, pl: Plan, H: int) -> np.ndarray:
+    """Reverse all-to-all of the GRADIENT of a replicated K/V tensor (see :func:`s2h_replicated`): the K/H local ranks
+    that received a copy of KV head h each hold the gradient contribution of their own query heads, so the gradient of
+    head h is their sum.  head [N,Bl,S,1,D] (fp64) -> [N,Bl,T,H,D]."""
+    head = np.ascontiguousarray(head)
+    N, Bl, S, one, D = head.shape
+    assert (N, Bl, S, one) == (pl.N, pl.Bl, pl.S, 1) and pl.K % H == 0 and H < pl.K
+    rep, T = pl.K // H, pl.T
+    out = np.zeros((N, Bl, T, H, D), dtype=head.dtype)
+    for g in range(pl.G):
+        for dst in range(pl.K):                    # owner of tokens [dst*T, (dst+1)*T)
+            for m in range(pl.K):                  # local rank that holds a copy of head m // rep
+                out[g * pl.K + dst, :, :, m // rep, :] += head[g * pl.K + m, :, dst * T:(dst + 1) * T, 0, :]
+    return out
+
+
 def h2s(head: np.ndarray, pl: Plan) -> np.ndarray:
     """Group-local all-to-all, head-sharded -> sequence-sharded (the reverse one)."""
     head = np.ascontiguousarray(head)
@@ -239,8 +255,11 @@ def layer_bwd(Xq, Xk, Xv, XdO, pl: Plan, scale: float | None = None, causal: boo
     """Backward of the sequence-parallel layer, step by step: partition the four global tensors,
     all-to-all each to head-sharded, per-rank attention backward, reverse all-to-all of dQ, dK, dV,
     collect.  Returns dict with head- and sequence-sharded gradients and the global ones."""
-    parts = [s2h(partition(X, pl), pl) for X in (Xq, Xk, Xv, XdO)]
-    qh, kh, vh, doh = parts
+    Hkv = Xk.shape[2]
+    replicated = Hkv % pl.K != 0                  # more ranks in a group than KV heads
+    kv_s2h = s2h_replicated if replicated else s2h
+    qh, doh = s2h(partition(Xq, pl), pl), s2h(partition(XdO, pl), pl)
+    kh, vh = kv_s2h(partition(Xk, pl), pl), kv_s2h(partition(Xv, pl), pl)
     dqh = np.empty(qh.shape, dtype=np.float64)
     dkh = np.empty(kh.shape, dtype=np.float64)
     dvh = np.empty(kh.shape, dtype=np.float64)
@@ -249,7 +268,7 @@ def layer_bwd(Xq, Xk, Xv, XdO, pl: Plan, scale: float | None = None, causal: boo
         dqh[r], dkh[r], dvh[r] = g["dQ"], g["dK"], g["dV"]
     out = dict(dq_head=dqh, dk_head=dkh, dv_head=dvh, do_head=doh)
     for n, a in (("dq", dqh), ("dk", dkh), ("dv", dvh)):
-        out[n + "_seq"] = h2s(a, pl)
+        out[n + "_seq"] = h2s_sum_replicated(a, pl, Hkv) if (replicated and n != "dq") else h2s(a, pl)
         out[n + "_global"] = gather(out[n + "_seq"], pl)
     return out
 

@@ -535,7 +535,7 @@ int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, 
         prm.dv[r] = (__nv_bfloat16 *)dv[r];
     }
     prm.n_ranks = pl->N; prm.Bl = pl->Bl; prm.S = pl->S; prm.Hq_l = pl->Hq_l; prm.Hkv_l = pl->Hkv_l;
-    prm.q_per_kv = pl->Hq / pl->Hkv; prm.causal = pl->causal;
+    prm.q_per_kv = pl->Hq_l / pl->Hkv_l; prm.causal = pl->causal;   // per rank (a replicated KV head serves all of a rank's query heads)
     prm.scale = scale == 0.f ? 1.f / sqrtf((float)pl->D) : scale;
     prm.scale_log2 = prm.scale * 1.4426950408889634f;
     prm.status = basp_status_device_ptr();
@@ -592,7 +592,7 @@ extern "C" int basp_attn_bwd(const basp_plan *pl, const void *const *q_head, con
     if (!pl || !q_head || !k_head || !v_head || !o_head || !do_head || !lse_shards || !dq_head || !dk_head ||
         !dv_head || !workspace)
         return BASP_ERR_NULL;
-    if (pl->D != 128 || pl->S % kT != 0 || pl->kv_rep != 1) return BASP_ERR_UNSUPPORTED;
+    if (pl->D != 128 || pl->S % kT != 0) return BASP_ERR_UNSUPPORTED;
     if (!aligned16(workspace)) return BASP_ERR_ALIGN;
     if (workspace_bytes < basp_attn_bwd_workspace_bytes(pl)) return BASP_ERR_WORKSPACE;
     for (int r = 0; r < pl->N; ++r) {

@@ -63,7 +63,7 @@ extern "C" int basp_layer_workspace_shards(const basp_plan *p, void *workspace, 
 extern "C" size_t basp_layer_bwd_workspace_bytes(const basp_plan *p) {
     if (!p) return 0;
     // head-sharded dO and dQ (query-sized), dK and dV (key-sized), then the attention-backward workspace
-    return (size_t)p->N * (2 * q_shard_bytes(p) + 2 * kv_shard_bytes(p)) + basp_attn_bwd_workspace_bytes(p);
+    return (size_t)p->N * (2 * q_shard_bytes(p) + 2 * kv_head_bytes(p)) + basp_attn_bwd_workspace_bytes(p);
 }
 
 extern "C" int basp_layer_bwd(const basp_plan *p, const void *const *q_head, const void *const *k_head,
@@ -76,7 +76,7 @@ extern "C" int basp_layer_bwd(const basp_plan *p, const void *const *q_head, con
     if (workspace_bytes < basp_layer_bwd_workspace_bytes(p)) return BASP_ERR_WORKSPACE;
     char *w = (char *)workspace;
     void *doh[BASP_MAX_RANKS], *dqh[BASP_MAX_RANKS], *dkh[BASP_MAX_RANKS], *dvh[BASP_MAX_RANKS];
-    const size_t qb = q_shard_bytes(p), kb = kv_shard_bytes(p);
+    const size_t qb = q_shard_bytes(p), kb = kv_head_bytes(p);
     for (int r = 0; r < p->N; ++r) {
         doh[r] = w + (size_t)r * qb;
         dqh[r] = w + (size_t)p->N * qb + (size_t)r * qb;

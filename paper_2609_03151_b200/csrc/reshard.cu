@@ -12,6 +12,8 @@
 //
 // HBM-bound: 2 bytes of traffic per byte of tensor, no arithmetic.  Each thread keeps U
 // independent 16-byte streaming loads in flight before its stores.
+#include <cuda_bf16.h>
+
 #include "common.cuh"
 
 namespace {
@@ -90,6 +92,32 @@ __global__ void __launch_bounds__(kThreads) reshard_kernel(const __grid_constant
         const uint32_t v = v0 + i * kThreads;
         if (v < t.shard_v) data[i] = ld_stream(kToHead ? seq + v : hp[i]);
     }
+    if (!kToHead && t.rep > 1) {
+        // The way back of a replicated tensor carries gradients: every copy holds the contribution of its own rank's
+        // query heads, the owner gets their sum (added in fp32, rounded to bf16 once).
+#pragma unroll
+        for (int i = 0; i < kUnroll; ++i) {
+            const uint32_t v = v0 + i * kThreads;
+            if (v >= t.shard_v) continue;
+            float acc[8];
+            const uint32_t w0[4] = {data[i].x, data[i].y, data[i].z, data[i].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { acc[2 * e] = __uint_as_float(w0[e] << 16); acc[2 * e + 1] = __uint_as_float(w0[e] & 0xffff0000u); }
+            for (uint32_t c = 1; c < t.rep; ++c) {
+                const uint4 d = ld_stream(reinterpret_cast<const uint4 *>(t.head[hrank[i] + c]) + hoff[i]);
+                const uint32_t wc[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) { acc[2 * e] += __uint_as_float(wc[e] << 16); acc[2 * e + 1] += __uint_as_float(wc[e] & 0xffff0000u); }
+            }
+            uint32_t o[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[2 * e], acc[2 * e + 1]);
+                o[e] = *reinterpret_cast<const uint32_t *>(&b2);
+            }
+            data[i] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+    }
 #pragma unroll
     for (int i = 0; i < kUnroll; ++i) {
         const uint32_t v = v0 + i * kThreads;
@@ -119,7 +147,6 @@ int fill_tensor(const basp_plan *p, const TensorArg &a, bool to_head, int r_begi
     // fewer heads than ranks in a group (KV heads under GQA): every head goes to K/H consecutive local ranks
     const int rep = a.n_heads % p->K == 0 ? 1 : (p->K % a.n_heads == 0 ? p->K / a.n_heads : 0);
     if (rep == 0) return BASP_ERR_INVALID;
-    if (rep > 1 && !to_head) return BASP_ERR_UNSUPPORTED;       // the way back would have to add the copies up
     const size_t run_bytes = (rep > 1 ? (size_t)1 : (size_t)(a.n_heads / p->K)) * p->D * 2;
     if (run_bytes % 16 != 0) return BASP_ERR_UNSUPPORTED;
     const size_t shard_bytes = (size_t)p->Bl * p->T * a.n_heads * p->D * 2;                 // sequence side

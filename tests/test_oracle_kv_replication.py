@@ -54,3 +54,28 @@ def test_replicated_equals_plain_exchange_when_heads_are_repeated():
     a = oracle.s2h_replicated(oracle.partition(Xk, pl), pl)
     b = oracle.s2h(oracle.partition(np.repeat(Xk, 2, axis=2), pl), pl)
     assert np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("N,B,Hq,Hkv", [(4, 1, 8, 2), (8, 2, 8, 1)])
+def test_backward_with_replication_equals_global_gradients(N, B, Hq, Hkv):
+    """dK and dV of a replicated KV head are the sums over its copies: the layer's gradients equal those of the
+    unpartitioned attention (oracle.attn_bwd on the global tensors, itself pinned by autograd and finite differences)."""
+    w = synth.Workload("r", N=N, B=B, S=64, Hq=Hq, Hkv=Hkv, D=16)
+    Xq, Xk, Xv = _inputs(w)
+    Xdo = synth.bits(synth.randn_bf16(__import__("torch").Generator().manual_seed(9), Xq.shape))
+    ref = oracle.attn_bwd(Xq, Xk, Xv, Xdo)
+    got = oracle.layer_bwd(Xq, Xk, Xv, Xdo, oracle.plan(N, B, w.S))
+    for n, k in (("dq", "dQ"), ("dk", "dK"), ("dv", "dV")):
+        assert np.abs(got[n + "_global"] - ref[k]).max() < 1e-12, n
+
+
+def test_sum_of_copies_is_the_adjoint_of_the_replicating_exchange():
+    """<s2h_replicated(x), y> = <x, h2s_sum_replicated(y)> for arbitrary x, y (the reverse exchange of a gradient is the
+    transpose of the forward exchange)."""
+    rng = np.random.default_rng(0)
+    pl = oracle.plan(8, 2, 32)
+    x = rng.standard_normal((8, pl.Bl, pl.T, 2, 4))
+    y = rng.standard_normal((8, pl.Bl, pl.S, 1, 4))
+    lhs = float((oracle.s2h_replicated(x, pl) * y).sum())
+    rhs = float((x * oracle.h2s_sum_replicated(y, pl, 2)).sum())
+    assert abs(lhs - rhs) < 1e-9 * max(1.0, abs(lhs))
