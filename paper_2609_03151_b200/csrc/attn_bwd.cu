@@ -48,6 +48,8 @@ struct BwdParams {
     const float *delta[R];
     __nv_bfloat16 *dk[R], *dv[R];
     int n_ranks, Bl, S, Hq_l, Hkv_l, q_per_kv, causal;
+    int Dg;                     // head dimension in memory (a multiple of 16 up to 128): the tile loads zero-fill the columns
+                                // past it, so every product is right as it stands; only the stores have to skip them
     float scale, scale_log2;
     int *status;
 };
@@ -229,7 +231,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             {
                 // quarters 0,1 write the two 64-column halves of dK, quarters 2,3 those of dV
                 __nv_bfloat16 *base = (g < 2 ? p.dk[item.r] : p.dv[item.r]) +
-                                      (((size_t)item.bl * p.S + (size_t)item.n * kT + row) * p.Hkv_l + item.hkv) * D +
+                                      (((size_t)item.bl * p.S + (size_t)item.n * kT + row) * p.Hkv_l + item.hkv) * p.Dg +
                                       64 * (g & 1);
                 const uint32_t col0 = (g < 2 ? kColDK : kColDV) + 64 * (g & 1);
 #pragma unroll
@@ -244,7 +246,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                         o4.y = pack_bf16x2(__uint_as_float(rr[8 * i + 2]), __uint_as_float(rr[8 * i + 3]));
                         o4.z = pack_bf16x2(__uint_as_float(rr[8 * i + 4]), __uint_as_float(rr[8 * i + 5]));
                         o4.w = pack_bf16x2(__uint_as_float(rr[8 * i + 6]), __uint_as_float(rr[8 * i + 7]));
-                        *reinterpret_cast<uint4 *>(base + cc * 32 + i * 8) = o4;
+                        if (64 * (g & 1) + cc * 32 + i * 8 < p.Dg) *reinterpret_cast<uint4 *>(base + cc * 32 + i * 8) = o4;
                     }
                 }
             }
@@ -308,6 +310,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                         const int row0 = item.bl * p.S + m * kT + wq * 32;
 #pragma unroll
                         for (int c = 0; c < 4; ++c)
+                            if (32 * c < p.Dg)          // a chunk wholly past the head dimension is padding
                             tma_reduce_add_3d(&p.dq_acc[item.r],
                                               (c < 2 ? sQ : sdO) + stage * kTileBytes + (c & 1) * 16384 + wq * 4096,
                                               32 * c, h, row0);
@@ -469,17 +472,17 @@ bwd_done:
 
 #undef BWD_WAIT
 
-// Delta[bl][h][s] = sum_d O[bl][s][h][d] * dO[bl][s][h][d]; one 16-lane group per (s, h) row of D = 128.
+// Delta[bl][h][s] = sum_d O[bl][s][h][d] * dO[bl][s][h][d]; one 16-lane group per (s, h) row of D <= 128.
 __global__ void __launch_bounds__(256) bwd_delta_kernel(const __nv_bfloat16 *__restrict__ o,
                                                         const __nv_bfloat16 *__restrict__ dout,
                                                         float *__restrict__ delta, int Bl, int S, int H, int D) {
-    const int lanes = D / 8;                            // threads per row (16 bytes each)
+    constexpr int lanes = 16;                           // threads per row (16 bytes each; D / 8 of them have data)
     const long long rows = (long long)Bl * S * H;
     const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long rowi = gid / lanes;
     const int part = (int)(gid % lanes);
     float acc = 0.f;
-    if (rowi < rows) {
+    if (rowi < rows && part * 8 < D) {
         const uint4 a = *reinterpret_cast<const uint4 *>(o + rowi * D + part * 8);
         const uint4 b = *reinterpret_cast<const uint4 *>(dout + rowi * D + part * 8);
         const uint32_t av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
@@ -535,6 +538,7 @@ int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, 
         prm.dv[r] = (__nv_bfloat16 *)dv[r];
     }
     prm.n_ranks = pl->N; prm.Bl = pl->Bl; prm.S = pl->S; prm.Hq_l = pl->Hq_l; prm.Hkv_l = pl->Hkv_l;
+    prm.Dg = pl->D;
     prm.q_per_kv = pl->Hq_l / pl->Hkv_l; prm.causal = pl->causal;   // per rank (a replicated KV head serves all of a rank's query heads)
     prm.scale = scale == 0.f ? 1.f / sqrtf((float)pl->D) : scale;
     prm.scale_log2 = prm.scale * 1.4426950408889634f;
@@ -542,7 +546,7 @@ int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, 
     if (!prm.status) return BASP_ERR_CUDA;
 
     BASP_CUDA_TRY(cudaMemsetAsync(acc0, 0, (size_t)pl->N * acc_b, st));
-    const long long row_threads = (long long)pl->Bl * pl->S * pl->Hq_l * (pl->D / 8);
+    const long long row_threads = (long long)pl->Bl * pl->S * pl->Hq_l * 16;
     for (int r = 0; r < pl->N; ++r) {
         bwd_delta_kernel<<<(unsigned)((row_threads + 255) / 256), 256, 0, st>>>(
             (const __nv_bfloat16 *)o[r], (const __nv_bfloat16 *)dout[r], const_cast<float *>(prm.delta[r]), pl->Bl,
@@ -592,7 +596,7 @@ extern "C" int basp_attn_bwd(const basp_plan *pl, const void *const *q_head, con
     if (!pl || !q_head || !k_head || !v_head || !o_head || !do_head || !lse_shards || !dq_head || !dk_head ||
         !dv_head || !workspace)
         return BASP_ERR_NULL;
-    if (pl->D != 128 || pl->S % kT != 0) return BASP_ERR_UNSUPPORTED;
+    if (pl->D < 16 || pl->D > 128 || pl->D % 16 != 0 || pl->S % kT != 0) return BASP_ERR_UNSUPPORTED;
     if (!aligned16(workspace)) return BASP_ERR_ALIGN;
     if (workspace_bytes < basp_attn_bwd_workspace_bytes(pl)) return BASP_ERR_WORKSPACE;
     for (int r = 0; r < pl->N; ++r) {
