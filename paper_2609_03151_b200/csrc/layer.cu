@@ -126,10 +126,10 @@ int get_pipe(HostPipe **out) {
 
 // Copies, kernels and read-backs are pipelined (three streams: copies in, the caller's stream for the kernels,
 // copies out).  The bus is the slow part, so the order of the copies is chosen to give the GPU its longest work
-// first: per group the K and V shards (a quarter of the bytes under GQA) go first, then the Q shards from the LAST
-// local rank down.  Under the causal mask the rows of local rank l cost (2l+1)/K^2 of the group's arithmetic, so
-// the launch for the last rank's rows - the longest - starts after K, V and one Q shard have arrived and the
-// shorter ones follow while the rest is still on the bus; O shard l is read back as soon as its launch is done.
+// first: a group's K and V shards (a quarter of the bytes under GQA) go ahead of its first Q shard, and the Q shards go
+// from the LAST local rank down, the groups taking turns.  Under the causal mask the rows of local rank l cost
+// (2l+1)/K^2 of the group's arithmetic, so the longest launches start first and the short ones follow while the
+// rest is still on the bus; O shard l is read back as soon as its launch is done.
 // Calls that overlap in time on one device share the internal streams and events: serialise them.
 extern "C" int basp_layer_fwd_host(const basp_plan *p, const void *const *q_seq_host, const void *const *k_seq_host,
                                    const void *const *v_seq_host, void *const *o_seq_host, void *device_arena,
@@ -155,24 +155,26 @@ extern "C" int basp_layer_fwd_host(const basp_plan *p, const void *const *q_seq_
     BASP_CUDA_TRY(cudaEventRecord(pipe->start, st));
     BASP_CUDA_TRY(cudaStreamWaitEvent(pipe->in, pipe->start, 0));
     BASP_CUDA_TRY(cudaStreamWaitEvent(pipe->out, pipe->start, 0));
-    for (int g = 0; g < p->G; ++g) {
-        const int r0 = g * p->K;
-        for (int l = 0; l < p->K; ++l) {
-            BASP_CUDA_TRY(cudaMemcpyAsync(kd[r0 + l], k_seq_host[r0 + l], kb, cudaMemcpyHostToDevice, pipe->in));
-            BASP_CUDA_TRY(cudaMemcpyAsync(vd[r0 + l], v_seq_host[r0 + l], kb, cudaMemcpyHostToDevice, pipe->in));
-        }
-        BASP_CUDA_TRY(cudaEventRecord(pipe->kv_arrived[g], pipe->in));
-        for (int l = p->K - 1; l >= 0; --l) {
-            BASP_CUDA_TRY(cudaMemcpyAsync(qd[r0 + l], q_seq_host[r0 + l], qb, cudaMemcpyHostToDevice, pipe->in));
-            BASP_CUDA_TRY(cudaEventRecord(pipe->arrived[r0 + l], pipe->in));
-        }
-    }
-    for (int g = 0; g < p->G; ++g) {
-        const int r0 = g * p->K;
-        BASP_CUDA_TRY(cudaStreamWaitEvent(st, pipe->kv_arrived[g], 0));
-        if (by_chunk) {
-            for (int l = p->K - 1; l >= 0; --l) {
-                BASP_CUDA_TRY(cudaStreamWaitEvent(st, pipe->arrived[r0 + l], 0));
+    if (by_chunk) {
+        // Units (group, local rank) in the order: every group's LAST local rank first (after that group's K and V), then
+        // the next-to-last of every group, and so on.  The longest launches are fed first and the groups alternate, so
+        // the GPU is not left waiting for the second group's shards while the first group's short launches finish.
+        for (int l = p->K - 1; l >= 0; --l)
+            for (int g = 0; g < p->G; ++g) {
+                const int r0 = g * p->K;
+                if (l == p->K - 1) {
+                    for (int j = 0; j < p->K; ++j) {
+                        BASP_CUDA_TRY(cudaMemcpyAsync(kd[r0 + j], k_seq_host[r0 + j], kb, cudaMemcpyHostToDevice, pipe->in));
+                        BASP_CUDA_TRY(cudaMemcpyAsync(vd[r0 + j], v_seq_host[r0 + j], kb, cudaMemcpyHostToDevice, pipe->in));
+                    }
+                }
+                BASP_CUDA_TRY(cudaMemcpyAsync(qd[r0 + l], q_seq_host[r0 + l], qb, cudaMemcpyHostToDevice, pipe->in));
+                BASP_CUDA_TRY(cudaEventRecord(pipe->arrived[r0 + l], pipe->in));
+            }
+        for (int l = p->K - 1; l >= 0; --l)
+            for (int g = 0; g < p->G; ++g) {
+                const int r0 = g * p->K;
+                BASP_CUDA_TRY(cudaStreamWaitEvent(st, pipe->arrived[r0 + l], 0));   // implies the group's K and V
                 const int range[4] = {r0, p->K, l * (p->T / 256), p->T / 256};
                 rc = basp_attn_dispatch_range(p, qd, kd, vd, od, nullptr, softmax_scale, true, range, stream);
                 if (rc != BASP_OK) return rc;
@@ -180,8 +182,19 @@ extern "C" int basp_layer_fwd_host(const basp_plan *p, const void *const *q_seq_
                 BASP_CUDA_TRY(cudaStreamWaitEvent(pipe->out, pipe->computed[r0 + l], 0));
                 BASP_CUDA_TRY(cudaMemcpyAsync(o_seq_host[r0 + l], od[r0 + l], qb, cudaMemcpyDeviceToHost, pipe->out));
             }
-        } else {
-            BASP_CUDA_TRY(cudaStreamWaitEvent(st, pipe->arrived[r0], 0));      // the Q shard sent last
+    } else {
+        for (int g = 0; g < p->G; ++g) {
+            const int r0 = g * p->K;
+            for (int l = 0; l < p->K; ++l) {
+                BASP_CUDA_TRY(cudaMemcpyAsync(kd[r0 + l], k_seq_host[r0 + l], kb, cudaMemcpyHostToDevice, pipe->in));
+                BASP_CUDA_TRY(cudaMemcpyAsync(vd[r0 + l], v_seq_host[r0 + l], kb, cudaMemcpyHostToDevice, pipe->in));
+                BASP_CUDA_TRY(cudaMemcpyAsync(qd[r0 + l], q_seq_host[r0 + l], qb, cudaMemcpyHostToDevice, pipe->in));
+            }
+            BASP_CUDA_TRY(cudaEventRecord(pipe->arrived[r0], pipe->in));
+        }
+        for (int g = 0; g < p->G; ++g) {
+            const int r0 = g * p->K;
+            BASP_CUDA_TRY(cudaStreamWaitEvent(st, pipe->arrived[r0], 0));
             const int range[4] = {r0, p->K, 0, (p->S / 128 + 1) / 2};
             rc = basp_attn_dispatch_range(p, qd, kd, vd, od, nullptr, softmax_scale, true, range, stream);
             if (rc != BASP_OK) return rc;
