@@ -261,13 +261,25 @@ def run_gpu(args, w: synth.Workload):
         for it in range(args.steps):
             basp.basp_out_proj(plan, hidden, o_seq, w_o, ys)
         pe[2].record()
+        ms_rope = None
+        if w.D in (64, 128):      # the same projection with rotary position embedding in its epilogue
+            cos, sin = (t.t().contiguous().to(dev) for t in synth.rope_tables(w.S, w.D))      # feature-major
+            re = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+            for it in range(args.warmup + args.steps):
+                if it == args.warmup:
+                    re[0].record()
+                basp.basp_qkv_proj_rope(plan, hidden, xs, w_qkv, cos, sin, q_seq, k_seq, v_seq)
+            re[1].record()
+            torch.cuda.synchronize()
+            ms_rope = re[0].elapsed_time(re[1]) / args.steps
         torch.cuda.synchronize()
         basp.basp_get_status()
         ms_qkv, ms_out = pe[0].elapsed_time(pe[1]) / args.steps, pe[1].elapsed_time(pe[2]) / args.steps
         f_qkv = 2.0 * N * Bl * T * hidden * (w.Hq + 2 * w.Hkv) * w.D
         f_out = 2.0 * N * Bl * T * hidden * w.Hq * w.D
         proj = {"hidden": hidden, "qkv_ms": ms_qkv, "qkv_tflops": f_qkv / ms_qkv / 1e9, "out_ms": ms_out,
-                "out_tflops": f_out / ms_out / 1e9, "peak_sustained": peaks["bf16_sustained"]}
+                "out_tflops": f_out / ms_out / 1e9, "qkv_rope_ms": ms_rope,
+                "qkv_rope_tflops": f_qkv / ms_rope / 1e9 if ms_rope else None, "peak_sustained": peaks["bf16_sustained"]}
         del xs, ys, w_qkv, w_o
 
     if args.quick:     # kernel timings only (what the ncu recipes in profiles/ run)

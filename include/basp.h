@@ -277,6 +277,15 @@ size_t basp_host_arena_bytes(const basp_plan *plan);
  * Hq*D, Hkv*D multiples of 256, else BASP_ERR_UNSUPPORTED.  Weights are shared by all ranks (one device pointer). */
 int basp_qkv_proj(const basp_plan *plan, int hidden, const void *const *x_seq, const void *w_qkv,
                   void *const *q_seq, void *const *k_seq, void *const *v_seq, void *stream);
+/* The QKV projection with rotary position embedding applied to Q and K in the epilogue (the paper does not treat
+ * position encodings; this is the rotate-half convention of the Llama / Qwen models it trains): within a head, feature
+ * j < D/2 pairs with feature j + D/2,  y_j = x_j cos - x_{j+D/2} sin,  y_{j+D/2} = x_{j+D/2} cos + x_j sin,  computed
+ * on the fp32 accumulators and rounded to bf16 once.  rope_cos / rope_sin: device fp32 tables [D/2][S], FEATURE-major
+ * (entry [j][pos]: the 128 rows of an output tile are consecutive positions, so this order reads whole lines), pos =
+ * the token's position in its sequence (local rank * T + row mod T).  V is not rotated.  Requires D = 64 or 128. */
+int basp_qkv_proj_rope(const basp_plan *plan, int hidden, const void *const *x_seq, const void *w_qkv,
+                       const float *rope_cos, const float *rope_sin, void *const *q_seq, void *const *k_seq,
+                       void *const *v_seq, void *stream);
 int basp_out_proj(const basp_plan *plan, int hidden, const void *const *o_seq, const void *w_o,
                   void *const *y_seq, void *stream);
 

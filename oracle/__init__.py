@@ -302,6 +302,32 @@ def linear(X: np.ndarray, W: np.ndarray) -> np.ndarray:
     return bf16_bits_to_f64(X) @ bf16_bits_to_f64(W).T
 
 
+def rope(x: np.ndarray, cos: np.ndarray, sin: np.ndarray, positions: np.ndarray) -> np.ndarray:
+    """Rotary position embedding in the rotate-half form, in fp64 (the paper does not treat position encodings; this
+    is the convention of the Llama / Qwen models it trains): within a head, feature j < D/2 pairs with feature
+    j + D/2 and the pair is turned by the angle of (position, j):
+        y_j = x_j cos - x_{j+D/2} sin,    y_{j+D/2} = x_{j+D/2} cos + x_j sin.
+    x [tokens, H, D] (fp64), cos / sin [S, D/2] tables (any float type, read as given), positions [tokens]."""
+    x = np.asarray(x, dtype=np.float64)
+    tokens, H, D = x.shape
+    half = D // 2
+    c = np.asarray(cos, dtype=np.float64)[np.asarray(positions)][:, None, :]      # [tokens, 1, D/2]
+    s_ = np.asarray(sin, dtype=np.float64)[np.asarray(positions)][:, None, :]
+    lo, hi = x[..., :half], x[..., half:]
+    return np.concatenate([lo * c - hi * s_, hi * c + lo * s_], axis=-1)
+
+
+def qkv_proj_rope(X: np.ndarray, W: np.ndarray, Hq: int, Hkv: int, D: int, cos, sin, positions) -> tuple:
+    """Q = X W_Q, K = X W_K, V = X W_V (Section II-A) with the rotation applied to Q and K before anything is rounded.
+    X [tokens, hidden], W [(Hq + 2 Hkv) D, hidden] as bf16 bits; returns fp64 (Q [tokens,Hq,D], K, V [tokens,Hkv,D])."""
+    Y = linear(X, W)
+    tokens = Y.shape[0]
+    q = Y[:, :Hq * D].reshape(tokens, Hq, D)
+    k = Y[:, Hq * D:(Hq + Hkv) * D].reshape(tokens, Hkv, D)
+    v = Y[:, (Hq + Hkv) * D:].reshape(tokens, Hkv, D)
+    return rope(q, cos, sin, positions), rope(k, cos, sin, positions), v
+
+
 # ----------------------------------------------------------------- bf16 helpers
 def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
     """Exact widening of bf16 bit patterns to fp64."""

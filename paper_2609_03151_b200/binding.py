@@ -31,6 +31,7 @@ EXPORTS = [
     "basp_layer_bwd", "basp_layer_bwd_workspace_bytes", "basp_get_status", "basp_clear_status",
     "basp_strerror", "basp_last_cuda_error", "basp_launch_count", "basp_selftest_wait_timeout", "basp_qkv_proj", "basp_out_proj",
     "basp_reshard_qkv_s2h_ranks", "basp_reshard_h2s_ranks", "basp_attn_fwd_ranks", "basp_layer_fwd_fused_ranks",
+    "basp_qkv_proj_rope",
 ]
 
 
@@ -84,6 +85,7 @@ lib.basp_clear_status.argtypes = [c_void_p]
 lib.basp_selftest_wait_timeout.argtypes = [ctypes.c_uint, c_void_p]
 lib.basp_qkv_proj.argtypes = [c_void_p, c_int, _PP, c_void_p, _PP, _PP, _PP, c_void_p]
 lib.basp_out_proj.argtypes = [c_void_p, c_int, _PP, c_void_p, _PP, c_void_p]
+lib.basp_qkv_proj_rope.argtypes = [c_void_p, c_int, _PP, c_void_p, c_void_p, c_void_p, _PP, _PP, _PP, c_void_p]
 lib.basp_strerror.argtypes = [c_int]
 lib.basp_strerror.restype = c_char_p
 lib.basp_last_cuda_error.restype = c_char_p
@@ -333,6 +335,13 @@ def basp_qkv_proj(plan, hidden, x_seq, w_qkv, q_seq, k_seq, v_seq, stream=None):
     n = plan.N
     _check(lib.basp_qkv_proj(plan.handle, int(hidden), _ptrs(x_seq, n), c_void_p(w_qkv.data_ptr()), _ptrs(q_seq, n),
                              _ptrs(k_seq, n), _ptrs(v_seq, n), _stream(stream)), "basp_qkv_proj")
+
+
+def basp_qkv_proj_rope(plan, hidden, x_seq, w_qkv, rope_cos, rope_sin, q_seq, k_seq, v_seq, stream=None):
+    n = plan.N
+    _check(lib.basp_qkv_proj_rope(plan.handle, int(hidden), _ptrs(x_seq, n), c_void_p(w_qkv.data_ptr()),
+                                  c_void_p(rope_cos.data_ptr()), c_void_p(rope_sin.data_ptr()), _ptrs(q_seq, n),
+                                  _ptrs(k_seq, n), _ptrs(v_seq, n), _stream(stream)), "basp_qkv_proj_rope")
 
 
 def basp_out_proj(plan, hidden, o_seq, w_o, y_seq, stream=None):

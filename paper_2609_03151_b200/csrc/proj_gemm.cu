@@ -36,6 +36,12 @@ struct GemmParams {
     int n_seg;
     int seg_begin[3], seg_ld[3];           // first output column of the segment; row pitch of its tensor (elements)
     __nv_bfloat16 *seg_ptr[3][R];
+    // rotary position embedding applied to the first `rope_segs` segments (Q, K) before the rounding to bf16:
+    // head dimension 2 * rope_half, tables [rope_half][rope_S] of cos and sin (feature-major: the 32 rows of a warp are
+    // 32 consecutive positions, so a warp's read of one feature is one 128-byte line), position of a row = the token's
+    // place in its sequence: local rank (r mod rope_K) * rope_T + row mod rope_T
+    int rope_segs, rope_half, rope_T, rope_K, rope_S;
+    const float *rope_cos, *rope_sin;
     int *status;
 };
 
@@ -135,6 +141,56 @@ __global__ void __launch_bounds__(kGemmThreads, 1) proj_gemm_kernel(const __grid
             __nv_bfloat16 *dst = p.seg_ptr[seg][r] + (size_t)grow * p.seg_ld[seg] + (n * kBN - p.seg_begin[seg]);
             GEMM_WAIT(&bars.acc_full[acc], (tile_cnt >> 1) & 1, 3, tile);
             tc_fence_after();
+            if (seg < p.rope_segs) {
+                // Rotate-half form: within a head, column j < D/2 pairs with column j + D/2:
+                //   y_j = x_j cos(t_j) - x_{j+D/2} sin(t_j),   y_{j+D/2} = x_{j+D/2} cos(t_j) + x_j sin(t_j),   t_j = pos * theta_j
+                // on the fp32 accumulators, one rounding to bf16 afterwards.  A thread owns a row, so both halves of every
+                // head of the tile are in its own TMEM lane.
+                const int half = p.rope_half, D2 = 2 * half;
+                const int pos = (r % p.rope_K) * p.rope_T + (grow % p.rope_T);
+                const float *ct = p.rope_cos + pos, *sn = p.rope_sin + pos;
+                for (int j0 = 0; j0 < half; j0 += 32) {
+                    // the angles depend on (position, feature) only: one fetch of 32 features serves every head of the tile
+                    float cv[32], sv[32];
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        const size_t off = (size_t)(j0 + e) * p.rope_S;
+                        cv[e] = __ldg(ct + off);
+                        sv[e] = __ldg(sn + off);
+                    }
+                    for (int hb = 0; hb < kBN; hb += D2) {
+                        uint32_t lo[32], hi[32];
+                        tmem_ld_x32(tmem + acc * kBN + hb + j0 + lane_addr, lo);
+                        tmem_ld_x32(tmem + acc * kBN + hb + half + j0 + lane_addr, hi);
+                        tmem_wait_ld();
+                        if (hb + D2 == kBN && j0 + 32 == half) {    // that was the last read of the accumulator
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&bars.acc_empty[acc]);
+                        }
+                        if (grow < p.M) {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                float yl[8], yh[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) {
+                                    const float xl = __uint_as_float(lo[8 * i + e]), xh = __uint_as_float(hi[8 * i + e]);
+                                    yl[e] = xl * cv[8 * i + e] - xh * sv[8 * i + e];
+                                    yh[e] = xh * cv[8 * i + e] + xl * sv[8 * i + e];
+                                }
+                                uint4 o4;
+                                o4.x = pack_bf16x2(yl[0], yl[1]); o4.y = pack_bf16x2(yl[2], yl[3]);
+                                o4.z = pack_bf16x2(yl[4], yl[5]); o4.w = pack_bf16x2(yl[6], yl[7]);
+                                *reinterpret_cast<uint4 *>(dst + hb + j0 + i * 8) = o4;
+                                o4.x = pack_bf16x2(yh[0], yh[1]); o4.y = pack_bf16x2(yh[2], yh[3]);
+                                o4.z = pack_bf16x2(yh[4], yh[5]); o4.w = pack_bf16x2(yh[6], yh[7]);
+                                *reinterpret_cast<uint4 *>(dst + hb + half + j0 + i * 8) = o4;
+                            }
+                        }
+                    }
+                }
+                continue;
+            }
 #pragma unroll
             for (int c = 0; c < kBN / 32; ++c) {
                 uint32_t rr[32];
@@ -178,9 +234,14 @@ struct Segment {
     void *const *ptrs;
 };
 
+struct Rope {
+    int segs;                 // leading segments to rotate (0 = none)
+    const float *cos, *sin;   // [D/2][S] each
+};
+
 template <int R>
 int gemm_launch(const basp_plan *pl, const void *const *a, const void *w, int M, int N, int K, const Segment *segs,
-                int n_seg, cudaStream_t st) {
+                int n_seg, const Rope &rope, cudaStream_t st) {
     GemmParams<R> prm;
     for (int r = 0; r < pl->N; ++r) {
         int rc = tmap::encode_rows_heads_d(&prm.a[r], a[r], (uint64_t)M, 1, (uint64_t)K, kBM);
@@ -196,6 +257,8 @@ int gemm_launch(const basp_plan *pl, const void *const *a, const void *w, int M,
         for (int r = 0; r < pl->N; ++r) prm.seg_ptr[s][r] = (__nv_bfloat16 *)segs[s].ptrs[r];
         col += segs[s].cols;
     }
+    prm.rope_segs = rope.segs; prm.rope_half = pl->D / 2; prm.rope_T = pl->T; prm.rope_K = pl->K; prm.rope_S = pl->S;
+    prm.rope_cos = rope.cos; prm.rope_sin = rope.sin;
     prm.status = basp_status_device_ptr();
     if (!prm.status) return BASP_ERR_CUDA;
     int dev = 0, sms = 0;
@@ -212,7 +275,7 @@ int gemm_launch(const basp_plan *pl, const void *const *a, const void *w, int M,
 }
 
 int gemm_dispatch(const basp_plan *pl, const void *const *a, const void *w, int N, int K, const Segment *segs, int n_seg,
-                  void *stream) {
+                  const Rope &rope, void *stream) {
     const int M = pl->Bl * pl->T;
     if (K <= 0 || K % kBK != 0) return BASP_ERR_UNSUPPORTED;
     for (int s = 0; s < n_seg; ++s)
@@ -229,8 +292,14 @@ int gemm_dispatch(const basp_plan *pl, const void *const *a, const void *w, int 
                 if (segs[s].ptrs[r] == a[r2] || segs[s].ptrs[r] == w) return BASP_ERR_ALIAS;
         }
     }
-    if (pl->N <= 8) return gemm_launch<8>(pl, a, w, M, N, K, segs, n_seg, (cudaStream_t)stream);
-    return gemm_launch<BASP_MAX_RANKS>(pl, a, w, M, N, K, segs, n_seg, (cudaStream_t)stream);
+    if (rope.segs > 0) {
+        // a head's two halves must be whole 32-column chunks of one tile: D = 64 or 128
+        if (pl->D != 64 && pl->D != 128) return BASP_ERR_UNSUPPORTED;
+        if (!rope.cos || !rope.sin) return BASP_ERR_NULL;
+        if (((uintptr_t)rope.cos & 3) || ((uintptr_t)rope.sin & 3)) return BASP_ERR_ALIGN;
+    }
+    if (pl->N <= 8) return gemm_launch<8>(pl, a, w, M, N, K, segs, n_seg, rope, (cudaStream_t)stream);
+    return gemm_launch<BASP_MAX_RANKS>(pl, a, w, M, N, K, segs, n_seg, rope, (cudaStream_t)stream);
 }
 
 }  // namespace
@@ -239,7 +308,16 @@ extern "C" int basp_qkv_proj(const basp_plan *plan, int hidden, const void *cons
                              void *const *q_seq, void *const *k_seq, void *const *v_seq, void *stream) {
     if (!plan) return BASP_ERR_NULL;
     const Segment segs[3] = {{plan->Hq * plan->D, q_seq}, {plan->Hkv * plan->D, k_seq}, {plan->Hkv * plan->D, v_seq}};
-    return gemm_dispatch(plan, x_seq, w_qkv, (plan->Hq + 2 * plan->Hkv) * plan->D, hidden, segs, 3, stream);
+    return gemm_dispatch(plan, x_seq, w_qkv, (plan->Hq + 2 * plan->Hkv) * plan->D, hidden, segs, 3, Rope{0, nullptr, nullptr}, stream);
+}
+
+extern "C" int basp_qkv_proj_rope(const basp_plan *plan, int hidden, const void *const *x_seq, const void *w_qkv,
+                                  const float *rope_cos, const float *rope_sin, void *const *q_seq, void *const *k_seq,
+                                  void *const *v_seq, void *stream) {
+    if (!plan) return BASP_ERR_NULL;
+    const Segment segs[3] = {{plan->Hq * plan->D, q_seq}, {plan->Hkv * plan->D, k_seq}, {plan->Hkv * plan->D, v_seq}};
+    return gemm_dispatch(plan, x_seq, w_qkv, (plan->Hq + 2 * plan->Hkv) * plan->D, hidden, segs, 3,
+                         Rope{2, rope_cos, rope_sin}, stream);
 }
 
 extern "C" int basp_out_proj(const basp_plan *plan, int hidden, const void *const *o_seq, const void *w_o,
@@ -247,5 +325,5 @@ extern "C" int basp_out_proj(const basp_plan *plan, int hidden, const void *cons
     if (!plan) return BASP_ERR_NULL;
     if (hidden <= 0) return BASP_ERR_INVALID;
     const Segment segs[1] = {{hidden, y_seq}};
-    return gemm_dispatch(plan, o_seq, w_o, hidden, plan->Hq * plan->D, segs, 1, stream);
+    return gemm_dispatch(plan, o_seq, w_o, hidden, plan->Hq * plan->D, segs, 1, Rope{0, nullptr, nullptr}, stream);
 }

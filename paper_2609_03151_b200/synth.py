@@ -114,3 +114,11 @@ def random_bits(shape, seed: int = 0) -> np.ndarray:
     """Arbitrary 16-bit patterns (for bit-exact permutation checks)."""
     rng = np.random.default_rng(seed)
     return rng.integers(0, 1 << 16, size=shape, dtype=np.uint16)
+
+
+def rope_tables(S: int, D: int, base: float = 500000.0):
+    """cos and sin of position * base^(-2j/D), j < D/2, as fp32 tensors [S, D/2] (angles formed in fp64; base 500000 is
+    Llama 3's).  The rotary variant of the QKV projection takes them transposed, [D/2, S] contiguous."""
+    j = torch.arange(D // 2, dtype=torch.float64)
+    ang = torch.arange(S, dtype=torch.float64)[:, None] * (base ** (-2.0 * j / D))[None, :]
+    return torch.cos(ang).to(torch.float32), torch.sin(ang).to(torch.float32)

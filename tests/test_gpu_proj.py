@@ -64,3 +64,47 @@ def test_projection_argument_checks(basp):
     with pytest.raises(basp.BaspError) as e:
         basp.basp_qkv_proj(pl, 100, x, wq, q, kv, kv)          # hidden not a multiple of 64
     assert e.value.code == basp.BASP_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("w,hidden", [
+    (synth.Workload("r1", N=2, B=2, S=256, Hq=4, Hkv=2, D=128), 512),
+    (synth.Workload("r2", N=4, B=1, S=800, Hq=8, Hkv=4, D=64), 320),        # one group of 4: positions run across ranks; T = 200
+    (synth.Workload("r3", N=2, B=4, S=192, Hq=4, Hkv=2, D=128, G=1), 256),   # several sequences per rank: positions restart
+])
+def test_qkv_projection_with_rope(basp, w, hidden):
+    """Rotary embedding in the GEMM epilogue against the oracle: rotation of the fp64 product, position of a row =
+    local rank * T + its token index inside the sequence chunk."""
+    pl = make_plan(basp, w)
+    op = oracle.plan(w.N, w.B, w.S, w.G)
+    g = torch.Generator().manual_seed(7 * w.S + hidden)
+    M = op.Bl * op.T
+    x = [synth.randn_bf16(g, (M, hidden)) for _ in range(w.N)]
+    w_qkv = (torch.randn(((w.Hq + 2 * w.Hkv) * w.D, hidden), generator=g) / hidden ** 0.5).to(torch.bfloat16)
+    cos, sin = synth.rope_tables(w.S, w.D)
+    dq = [torch.full((op.Bl, op.T, w.Hq, w.D), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(w.N)]
+    dk = [torch.full((op.Bl, op.T, w.Hkv, w.D), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(w.N)]
+    dv = [torch.full_like(t, float("nan")) for t in dk]
+    basp.basp_clear_status()
+    basp.basp_qkv_proj_rope(pl, hidden, [t.cuda() for t in x], w_qkv.cuda(), cos.t().contiguous().cuda(),
+                            sin.t().contiguous().cuda(), dq, dk, dv)      # the call takes the tables feature-major
+    basp.basp_get_status()
+    for r in range(w.N):
+        info = op.rank_info(r, w.Hq, w.Hkv)
+        pos = np.tile(np.arange(info["token_begin"], info["token_end"]), op.Bl)      # row bl*T + t -> position l*T + t
+        q, k, v = oracle.qkv_proj_rope(synth.bits(x[r]), synth.bits(w_qkv), w.Hq, w.Hkv, w.D, cos.numpy(), sin.numpy(), pos)
+        f = lambda t, h: t.float().cpu().numpy().astype(np.float64).reshape(M, h, w.D)
+        close(f(dq[r], w.Hq), q, "Q"); close(f(dk[r], w.Hkv), k, "K"); close(f(dv[r], w.Hkv), v, "V")
+
+
+def test_rope_argument_checks(basp):
+    w = synth.Workload("re", N=2, B=2, S=256, Hq=4, Hkv=2, D=96)
+    pl = make_plan(basp, w)
+    x = [torch.zeros((128, 256), dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    wq = torch.zeros(((4 + 4) * 96, 256), dtype=torch.bfloat16, device="cuda")
+    q = [torch.zeros((1, 128, 4, 96), dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    k = [torch.zeros((1, 128, 2, 96), dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    v = [torch.zeros_like(t) for t in k]
+    cs = torch.zeros((48, 256), dtype=torch.float32, device="cuda")
+    with pytest.raises(basp.BaspError) as e:
+        basp.basp_qkv_proj_rope(pl, 256, x, wq, cs, cs, q, k, v)
+    assert e.value.code == basp.BASP_ERR_UNSUPPORTED          # D = 96: a head's halves are not whole 32-column chunks
