@@ -223,7 +223,7 @@ int basp_layer_workspace_shards(const basp_plan *plan, void *workspace, void **q
  * [Bl][S][Hq/K][D]; k, v, dk, dv [Bl][S][Hkv/K][D]; lse as written by the forward.  bf16 in and out,
  * fp32 accumulation; dQ is accumulated with floating-point atomics, so its last bits may differ
  * between runs.  Requires D a multiple of 16 up to 128 (the kernel is 128 columns wide: a smaller D runs with the
- * missing columns zero-filled by the tile loads and costs the same time as D = 128) and S a multiple of 128.  `workspace`: device memory of at least
+ * missing columns zero-filled by the tile loads and costs the same time as D = 128); S is arbitrary (ragged last tiles are masked).  `workspace`: device memory of at least
  * basp_attn_bwd_workspace_bytes(plan) bytes (fp32 dQ accumulator and Delta). */
 int basp_attn_bwd(const basp_plan *plan, const void *const *q_head, const void *const *k_head,
                   const void *const *v_head, const void *const *o_head, const void *const *do_head,

@@ -23,6 +23,8 @@
 #include <cuda.h>
 #include <math.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 #include "ptx.cuh"
 #include "tmap.cuh"
@@ -60,7 +62,7 @@ struct BwdItem {
 
 template <int R>
 __device__ __forceinline__ bool bwd_get_item(const BwdParams<R> &p, int round, BwdItem &it) {
-    const int n_kt = p.S / kT;
+    const int n_kt = (p.S + kT - 1) / kT;      // the last tile may be ragged
     const int streams = p.n_ranks * p.Bl * p.Hkv_l;
     const int total = n_kt * streams;
     const int pos = (round & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x;
@@ -183,25 +185,43 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     tmem_wait_ld();
                     BPH_T(t2);
                     const bool diag = p.causal && m == item.n;
+                    // A ragged last tile (S is not a multiple of 128) holds rows of the next sequence of the shard, or TMA
+                    // zero fill, past the end: those keys and queries take no part (P = 0 makes dS = 0 and with it every
+                    // contribution to dV, dQ, dK).
+                    // Folded into one column window per thread: this thread's columns c (query 32g + c) count iff
+                    // c_lo <= c < c_hi.  Only edge steps (the diagonal, a ragged last tile) carry the test at all: the loop
+                    // is instantiated twice so that the common step has no masking code.
+                    const bool edge = diag || (m + 1) * kT > p.S || (item.n + 1) * kT > p.S;
+                    int c_lo = 0, c_hi = 32;
+                    if (edge) {
+                        if (diag) c_lo = row - 32 * g;                              // queries earlier than key `row`
+                        if (item.n * kT + row >= p.S) c_lo = 32;                    // this thread's key row does not exist
+                        if (p.S - m * kT - 32 * g < c_hi) c_hi = p.S - m * kT - 32 * g;   // queries past the end
+                    }
                     const float *lse_b = s_lse + buf * kT + 32 * g;
                     const float *del_b = s_delta + buf * kT + 32 * g;
+                    auto p_and_ds = [&](auto edge_tag) {
+                        constexpr bool kEdge = decltype(edge_tag)::value;
 #pragma unroll
-                    for (int c = 0; c < 32; c += 4) {
-                        const float4 l4 = *reinterpret_cast<const float4 *>(lse_b + c);
-                        const float4 d4 = *reinterpret_cast<const float4 *>(del_b + c);
-                        const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dl[4] = {d4.x, d4.y, d4.z, d4.w};
-                        float pv[4], dsv[4];
+                        for (int c = 0; c < 32; c += 4) {
+                            const float4 l4 = *reinterpret_cast<const float4 *>(lse_b + c);
+                            const float4 d4 = *reinterpret_cast<const float4 *>(del_b + c);
+                            const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dl[4] = {d4.x, d4.y, d4.z, d4.w};
+                            float pv[4], dsv[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            pv[e] = exp2_approx(fmaf(__uint_as_float(st[c + e]), p.scale_log2, -lv[e]));
-                            if (diag && 32 * g + c + e < row) pv[e] = 0.f;   // query 32g+c+e is earlier than key `row`
-                            dsv[e] = pv[e] * (__uint_as_float(dp[c + e]) - dl[e]) * p.scale;
+                            for (int e = 0; e < 4; ++e) {
+                                pv[e] = exp2_approx(fmaf(__uint_as_float(st[c + e]), p.scale_log2, -lv[e]));
+                                if (kEdge && (c + e < c_lo || c + e >= c_hi)) pv[e] = 0.f;
+                                dsv[e] = pv[e] * (__uint_as_float(dp[c + e]) - dl[e]) * p.scale;
+                            }
+                            st[c >> 1] = pack_bf16x2(pv[0], pv[1]);
+                            st[(c >> 1) + 1] = pack_bf16x2(pv[2], pv[3]);
+                            dp[c >> 1] = pack_bf16x2(dsv[0], dsv[1]);
+                            dp[(c >> 1) + 1] = pack_bf16x2(dsv[2], dsv[3]);
                         }
-                        st[c >> 1] = pack_bf16x2(pv[0], pv[1]);
-                        st[(c >> 1) + 1] = pack_bf16x2(pv[2], pv[3]);
-                        dp[c >> 1] = pack_bf16x2(dsv[0], dsv[1]);
-                        dp[(c >> 1) + 1] = pack_bf16x2(dsv[2], dsv[3]);
-                    }
+                    };
+                    if (edge) p_and_ds(std::true_type{});
+                    else p_and_ds(std::false_type{});
                     BPH_T(t3);
                     // P^T (bf16) over this quarter's own score columns: TMEM columns 32g .. 32g+15
                     tmem_st_x16(tmem + kColST + 32 * g + lane_addr, *reinterpret_cast<const uint32_t(*)[16]>(&st[0]));
@@ -246,7 +266,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                         o4.y = pack_bf16x2(__uint_as_float(rr[8 * i + 2]), __uint_as_float(rr[8 * i + 3]));
                         o4.z = pack_bf16x2(__uint_as_float(rr[8 * i + 4]), __uint_as_float(rr[8 * i + 5]));
                         o4.w = pack_bf16x2(__uint_as_float(rr[8 * i + 6]), __uint_as_float(rr[8 * i + 7]));
-                        if (64 * (g & 1) + cc * 32 + i * 8 < p.Dg) *reinterpret_cast<uint4 *>(base + cc * 32 + i * 8) = o4;
+                        if (64 * (g & 1) + cc * 32 + i * 8 < p.Dg && item.n * kT + row < p.S)
+                            *reinterpret_cast<uint4 *>(base + cc * 32 + i * 8) = o4;
                     }
                 }
             }
@@ -357,8 +378,21 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     {   // row statistics of the query tile: LSE (to log2 units) and Delta, four rows per lane.  The buffer
                         // has the stage's parity: its last readers (step it-2) finished before the stage was released.
                         const size_t off = ((size_t)item.bl * p.Hq_l + h) * p.S + (size_t)m * kT + 4 * lane;
-                        float4 l4 = *reinterpret_cast<const float4 *>(p.lse[item.r] + off);
-                        const float4 d4 = *reinterpret_cast<const float4 *>(p.delta[item.r] + off);
+                        float4 l4, d4;
+                        if ((p.S & 3) == 0 && (m + 1) * kT <= p.S) {
+                            l4 = *reinterpret_cast<const float4 *>(p.lse[item.r] + off);
+                            d4 = *reinterpret_cast<const float4 *>(p.delta[item.r] + off);
+                        } else {                       // ragged: rows of (bl, h) are not 16-byte aligned, or the tile runs past S
+                            float lv[4], dv4[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const bool in_seq = m * kT + 4 * lane + e < p.S;
+                                lv[e] = in_seq ? p.lse[item.r][off + e] : 0.f;
+                                dv4[e] = in_seq ? p.delta[item.r][off + e] : 0.f;
+                            }
+                            l4 = make_float4(lv[0], lv[1], lv[2], lv[3]);
+                            d4 = make_float4(dv4[0], dv4[1], dv4[2], dv4[3]);
+                        }
                         l4.x *= 1.4426950408889634f; l4.y *= 1.4426950408889634f;
                         l4.z *= 1.4426950408889634f; l4.w *= 1.4426950408889634f;
                         *reinterpret_cast<float4 *>(s_lse + stage * kT + 4 * lane) = l4;
@@ -557,7 +591,7 @@ int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, 
     int dev = 0, sms = 0;
     BASP_CUDA_TRY(cudaGetDevice(&dev));
     BASP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    const long long items = (long long)(pl->S / kT) * pl->N * pl->Bl * pl->Hkv_l;
+    const long long items = (long long)((pl->S + kT - 1) / kT) * pl->N * pl->Bl * pl->Hkv_l;
     const int grid = (int)(items < sms ? items : sms);
     const int smem = 7 * kT * 128 * 2 + 4 * kT * (int)sizeof(float) + (int)sizeof(BwdBars);
     BASP_CUDA_TRY(cudaFuncSetAttribute(attn_bwd_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
@@ -596,7 +630,7 @@ extern "C" int basp_attn_bwd(const basp_plan *pl, const void *const *q_head, con
     if (!pl || !q_head || !k_head || !v_head || !o_head || !do_head || !lse_shards || !dq_head || !dk_head ||
         !dv_head || !workspace)
         return BASP_ERR_NULL;
-    if (pl->D < 16 || pl->D > 128 || pl->D % 16 != 0 || pl->S % kT != 0) return BASP_ERR_UNSUPPORTED;
+    if (pl->D < 16 || pl->D > 128 || pl->D % 16 != 0) return BASP_ERR_UNSUPPORTED;
     if (!aligned16(workspace)) return BASP_ERR_ALIGN;
     if (workspace_bytes < basp_attn_bwd_workspace_bytes(pl)) return BASP_ERR_WORKSPACE;
     for (int r = 0; r < pl->N; ++r) {

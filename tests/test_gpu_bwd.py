@@ -65,6 +65,17 @@ def test_attn_bwd_matches_oracle(basp, name, w):
         assert_grad_close(g, r, f"{name} {n}")
 
 
+@pytest.mark.parametrize("S,causal", [(200, True), (333, True), (1000, True), (77, False), (129, True)])
+def test_attn_bwd_ragged_sequence_lengths(basp, S, causal):
+    """S not a multiple of the 128-row tile, two sequences per rank: what follows a ragged end is the next sequence (its
+    rows must neither be read into the gradients nor be written), and the LSE / Delta rows are not 16-byte aligned."""
+    w = synth.Workload("ragged_S", N=2, B=4, S=S, Hq=4, Hkv=2, D=128, G=2)
+    got, ref = run_attn_bwd(basp, w, causal=causal, seed=S)
+    for g, r, n in zip(got, ref, ("dQ", "dK", "dV")):
+        assert np.isfinite(g).all(), f"S={S} {n}: not fully written"
+        assert_grad_close(g, r, f"S={S} {n}")
+
+
 def test_attn_bwd_noncausal(basp):
     w = synth.Workload("nc", N=2, B=2, S=256, Hq=2, Hkv=1, D=128)
     got, ref = run_attn_bwd(basp, w, causal=False, seed=3)
