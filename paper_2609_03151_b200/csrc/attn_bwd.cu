@@ -212,7 +212,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                             for (int e = 0; e < 4; ++e) {
                                 pv[e] = exp2_approx(fmaf(__uint_as_float(st[c + e]), p.scale_log2, -lv[e]));
                                 if (kEdge && (c + e < c_lo || c + e >= c_hi)) pv[e] = 0.f;
-                                dsv[e] = pv[e] * (__uint_as_float(dp[c + e]) - dl[e]) * p.scale;
+                                dsv[e] = pv[e] * fmaf(__uint_as_float(dp[c + e]), p.scale, dl[e]);   // dl = -Delta scale
                             }
                             st[c >> 1] = pack_bf16x2(pv[0], pv[1]);
                             st[(c >> 1) + 1] = pack_bf16x2(pv[2], pv[3]);
@@ -395,6 +395,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                         }
                         l4.x *= 1.4426950408889634f; l4.y *= 1.4426950408889634f;
                         l4.z *= 1.4426950408889634f; l4.w *= 1.4426950408889634f;
+                        d4.x *= -p.scale; d4.y *= -p.scale; d4.z *= -p.scale; d4.w *= -p.scale;   // staged as -Delta scale
                         *reinterpret_cast<float4 *>(s_lse + stage * kT + 4 * lane) = l4;
                         *reinterpret_cast<float4 *>(s_delta + stage * kT + 4 * lane) = d4;
                         __syncwarp();
