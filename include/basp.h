@@ -238,6 +238,17 @@ int basp_reshard_grads_h2s(const basp_plan *plan, const void *const *dq_head, co
                            const void *const *dv_head, void *const *dq_seq, void *const *dk_seq,
                            void *const *dv_seq, void *stream);
 
+/* ---- backward of the whole layer from SEQUENCE-sharded activations: for a forward pass that kept no head-sharded
+ * copies (basp_layer_fwd_fused).  The all-to-alls of Q, K, V, O and dO are redone here (two launches), then the
+ * attention backward and the reverse all-to-alls of the gradients.  lse_shards: as written by the forward.  `workspace`
+ * of at least basp_layer_bwd_seq_workspace_bytes(plan) bytes holds the head-sharded Q, K, V, O, dO, dQ, dK, dV and the
+ * attention-backward workspace. */
+int basp_layer_bwd_seq(const basp_plan *plan, const void *const *q_seq, const void *const *k_seq,
+                       const void *const *v_seq, const void *const *o_seq, const float *const *lse_shards,
+                       const void *const *do_seq, void *const *dq_seq, void *const *dk_seq, void *const *dv_seq,
+                       void *workspace, size_t workspace_bytes, float softmax_scale, void *stream);
+size_t basp_layer_bwd_seq_workspace_bytes(const basp_plan *plan);
+
 /* ---- backward of the whole layer: all-to-all of dO (sequence- to head-sharded), attention
  * backward on the saved head-sharded Q, K, V, O and LSE of the forward, reverse all-to-alls of
  * dQ, dK, dV.  do_seq / dq_seq / dk_seq / dv_seq are SEQUENCE-sharded.  `workspace` of at least

@@ -31,7 +31,7 @@ EXPORTS = [
     "basp_layer_bwd", "basp_layer_bwd_workspace_bytes", "basp_get_status", "basp_clear_status",
     "basp_strerror", "basp_last_cuda_error", "basp_launch_count", "basp_selftest_wait_timeout", "basp_qkv_proj", "basp_out_proj",
     "basp_reshard_qkv_s2h_ranks", "basp_reshard_h2s_ranks", "basp_attn_fwd_ranks", "basp_layer_fwd_fused_ranks",
-    "basp_qkv_proj_rope",
+    "basp_qkv_proj_rope", "basp_layer_bwd_seq", "basp_layer_bwd_seq_workspace_bytes",
 ]
 
 
@@ -73,7 +73,8 @@ lib.basp_layer_workspace_shards.argtypes = [c_void_p, c_void_p] + [_PP] * 4
 lib.basp_attn_bwd.argtypes = [c_void_p] + [_PP] * 9 + [c_void_p, c_size_t, c_float, c_void_p]
 lib.basp_reshard_grads_h2s.argtypes = [c_void_p] + [_PP] * 6 + [c_void_p]
 lib.basp_layer_bwd.argtypes = [c_void_p] + [_PP] * 9 + [c_void_p, c_size_t, c_float, c_void_p]
-for _n in ("basp_attn_bwd_workspace_bytes", "basp_layer_bwd_workspace_bytes"):
+lib.basp_layer_bwd_seq.argtypes = [c_void_p] + [_PP] * 9 + [c_void_p, c_size_t, c_float, c_void_p]
+for _n in ("basp_attn_bwd_workspace_bytes", "basp_layer_bwd_workspace_bytes", "basp_layer_bwd_seq_workspace_bytes"):
     getattr(lib, _n).argtypes = [c_void_p]
     getattr(lib, _n).restype = c_size_t
 lib.basp_workspace_bytes.argtypes = [c_void_p]
@@ -307,6 +308,19 @@ def basp_reshard_grads_h2s(plan, dq_head, dk_head, dv_head, dq_seq, dk_seq, dv_s
     _check(lib.basp_reshard_grads_h2s(plan.handle, *[_ptrs(t, n) for t in (dq_head, dk_head, dv_head, dq_seq, dk_seq,
                                                                            dv_seq)], _stream(stream)),
            "basp_reshard_grads_h2s")
+
+
+def basp_layer_bwd_seq_workspace_bytes(plan) -> int:
+    return int(lib.basp_layer_bwd_seq_workspace_bytes(plan.handle))
+
+
+def basp_layer_bwd_seq(plan, q_seq, k_seq, v_seq, o_seq, lse_shards, do_seq, dq_seq, dk_seq, dv_seq, workspace,
+                       softmax_scale=0.0, stream=None):
+    n = plan.N
+    _check(lib.basp_layer_bwd_seq(plan.handle, *[_ptrs(t, n) for t in (q_seq, k_seq, v_seq, o_seq, lse_shards, do_seq,
+                                                                       dq_seq, dk_seq, dv_seq)],
+                                  c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size(),
+                                  softmax_scale, _stream(stream)), "basp_layer_bwd_seq")
 
 
 def basp_layer_bwd(plan, q_head, k_head, v_head, o_head, lse_shards, do_seq, dq_seq, dk_seq, dv_seq, workspace,

@@ -92,6 +92,48 @@ extern "C" int basp_layer_bwd(const basp_plan *p, const void *const *q_head, con
     return basp_reshard_grads_h2s(p, dqh, dkh, dvh, dq_seq, dk_seq, dv_seq, stream);
 }
 
+extern "C" size_t basp_layer_bwd_seq_workspace_bytes(const basp_plan *p) {
+    if (!p) return 0;
+    // head-sharded Q, O, dO, dQ (query-sized), K, V, dK, dV (key-sized), then the attention-backward workspace
+    return (size_t)p->N * (4 * q_shard_bytes(p) + 4 * kv_head_bytes(p)) + basp_attn_bwd_workspace_bytes(p);
+}
+
+extern "C" int basp_layer_bwd_seq(const basp_plan *p, const void *const *q_seq, const void *const *k_seq,
+                                  const void *const *v_seq, const void *const *o_seq, const float *const *lse_shards,
+                                  const void *const *do_seq, void *const *dq_seq, void *const *dk_seq,
+                                  void *const *dv_seq, void *workspace, size_t workspace_bytes, float softmax_scale,
+                                  void *stream) {
+    if (!p || !workspace) return BASP_ERR_NULL;
+    if (!aligned16(workspace)) return BASP_ERR_ALIGN;
+    if (workspace_bytes < basp_layer_bwd_seq_workspace_bytes(p)) return BASP_ERR_WORKSPACE;
+    char *w = (char *)workspace;
+    void *qh[BASP_MAX_RANKS], *kh[BASP_MAX_RANKS], *vh[BASP_MAX_RANKS], *oh[BASP_MAX_RANKS], *doh[BASP_MAX_RANKS],
+        *dqh[BASP_MAX_RANKS], *dkh[BASP_MAX_RANKS], *dvh[BASP_MAX_RANKS];
+    const size_t qb = q_shard_bytes(p), kb = kv_head_bytes(p);
+    const size_t n = (size_t)p->N;
+    for (int r = 0; r < p->N; ++r) {
+        qh[r] = w + (size_t)r * qb;
+        oh[r] = w + n * qb + (size_t)r * qb;
+        doh[r] = w + n * 2 * qb + (size_t)r * qb;
+        dqh[r] = w + n * 3 * qb + (size_t)r * qb;
+        kh[r] = w + n * 4 * qb + (size_t)r * kb;
+        vh[r] = w + n * (4 * qb + kb) + (size_t)r * kb;
+        dkh[r] = w + n * (4 * qb + 2 * kb) + (size_t)r * kb;
+        dvh[r] = w + n * (4 * qb + 3 * kb) + (size_t)r * kb;
+    }
+    char *bwd_ws = w + n * (4 * qb + 4 * kb);
+    int rc = basp_reshard_qkv_s2h(p, q_seq, k_seq, v_seq, qh, kh, vh, stream);
+    if (rc != BASP_OK) return rc;
+    rc = basp_reshard_s2h(p, p->Hq, o_seq, oh, stream);
+    if (rc != BASP_OK) return rc;
+    rc = basp_reshard_s2h(p, p->Hq, do_seq, doh, stream);
+    if (rc != BASP_OK) return rc;
+    rc = basp_attn_bwd(p, qh, kh, vh, oh, doh, lse_shards, dqh, dkh, dvh, bwd_ws, workspace_bytes - (size_t)(bwd_ws - w),
+                       softmax_scale, stream);
+    if (rc != BASP_OK) return rc;
+    return basp_reshard_grads_h2s(p, dqh, dkh, dvh, dq_seq, dk_seq, dv_seq, stream);
+}
+
 namespace {
 // Copy streams and events of the host-buffer entry, created once per device (no device memory).
 struct HostPipe {

@@ -165,3 +165,28 @@ def test_full_size_train_step_sampled(basp):
     got_dv = gv[kvh // Hkl][0, w.S - ncols:, kvh % Hkl].float().cpu().numpy().astype(np.float64)
     assert_grad_close(got_dk, ref_dk, "config 5 dK tail")
     assert_grad_close(got_dv, ref_dv, "config 5 dV tail")
+
+
+@pytest.mark.parametrize("w", [
+    synth.shrink(synth.WORKLOADS["llama3_8b_128k_train"], 128),
+    synth.Workload("two_groups_rep", N=8, B=2, S=512, Hq=8, Hkv=2, D=64),          # replicated KV heads, D = 64
+], ids=lambda w: w.name)
+def test_fused_forward_then_backward_from_sequence_shards(basp, w):
+    """Forward through the fused kernel (no head-sharded copies exist), backward through basp_layer_bwd_seq, which redoes
+    the exchanges; against the oracle's layer backward."""
+    (Xq, Xk, Xv, Xdo), op = inputs(w, seed=2)
+    ref = oracle.layer_bwd(Xq, Xk, Xv, Xdo, op)
+    pl = make_plan(basp, w)
+    qs, ks, vs, dos = (to_dev(oracle.partition(X, op)) for X in (Xq, Xk, Xv, Xdo))
+    o = [torch.zeros_like(t) for t in qs]
+    lse = [torch.zeros((op.Bl, pl.Hq_l, w.S), dtype=torch.float32, device="cuda") for _ in range(w.N)]
+    basp.basp_clear_status()
+    basp.basp_layer_fwd_fused(pl, qs, ks, vs, o, lse)
+    gq = [torch.full_like(t, float("nan")) for t in qs]
+    gk = [torch.full_like(t, float("nan")) for t in ks]
+    gv = [torch.full_like(t, float("nan")) for t in ks]
+    ws = torch.empty(basp.basp_layer_bwd_seq_workspace_bytes(pl), dtype=torch.uint8, device="cuda")
+    basp.basp_layer_bwd_seq(pl, qs, ks, vs, o, lse, dos, gq, gk, gv, ws)
+    basp.basp_get_status()
+    for g, n in ((gq, "dq_seq"), (gk, "dk_seq"), (gv, "dv_seq")):
+        assert_grad_close(to_f64(g), ref[n], n)
