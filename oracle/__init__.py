@@ -68,6 +68,15 @@ class Plan:
     Bl: int     # sequences per group
     S: int      # tokens per sequence
     T: int      # tokens per rank and sequence
+    T_last: int = 0   # tokens of a group's LAST rank when K does not divide S (plan_uneven); 0 = T
+
+    @property
+    def uneven(self) -> bool:
+        return self.T_last not in (0, self.T)
+
+    def token_range(self, l: int) -> tuple[int, int]:
+        """Tokens [begin, end) of local rank l (Algorithm 2's token_start / token_end, clipped to the sequence)."""
+        return min(l * self.T, self.S), min((l + 1) * self.T, self.S)
 
     def group_ranks(self, g: int) -> list[int]:
         out = (ctypes.c_int * self.K)()
@@ -93,6 +102,20 @@ def plan(N: int, B: int, S: int, G: int = 0) -> Plan:
     return Plan(N=N, B=B, G=G_, K=K, Bl=Bl, S=S, T=T)
 
 
+def plan_uneven(N: int, B: int, S: int, G: int = 0) -> Plan:
+    """The plan for a sequence length that the group size does not divide.  Algorithm 2 writes the chunk as L / K and
+    the paper says nothing about a remainder; the reading taken: chunk = ceil(S / K), local rank l holds tokens
+    [l chunk, min((l+1) chunk, S)), so only the group's last rank is short, and it must not be empty.  The groups
+    themselves (Algorithm 1) do not depend on S."""
+    base = plan(N, B, N, G)                      # group structure only (any S that K divides)
+    K = base.K
+    T = -(-S // K)
+    T_last = S - (K - 1) * T
+    if S <= 0 or T_last <= 0:
+        raise ValueError(f"invalid uneven plan N={N} B={B} G={G} S={S}: the last rank of a group would be empty")
+    return Plan(N=N, B=B, G=base.G, K=K, Bl=base.Bl, S=S, T=T, T_last=T_last)
+
+
 # ------------------------------------------------------------------ permutations
 def _esize(a: np.ndarray) -> int:
     return int(a.dtype.itemsize)
@@ -114,6 +137,73 @@ def gather(shards: np.ndarray, pl: Plan) -> np.ndarray:
     N, Bl, T, H, D = shards.shape
     out = np.empty((pl.B, pl.S, H, D), dtype=shards.dtype)
     _load().oracle_gather(_p(shards), _p(out), pl.N, pl.K, pl.Bl, pl.S, H, D, _esize(shards))
+    return out
+
+
+# The same four maps when the last rank of a group is short (plan_uneven): the shards differ in length, so they are a
+# list of N arrays [Bl, T_r, H, D]; the head-sharded side is unchanged ([N, Bl, S, H/K, D], every rank holds whole
+# sequences).  Written as slice assignments of the index maps, one (group, source rank, destination rank) at a time.
+def partition_uneven(X: np.ndarray, pl: Plan) -> list:
+    """Algorithm 2 for every rank with chunk = ceil(S/K): rank gK+l gets X[g Bl:(g+1) Bl, token_range(l)]."""
+    assert X.shape[0] == pl.B and X.shape[1] == pl.S
+    out = []
+    for r in range(pl.N):
+        g, l = divmod(r, pl.K)
+        t0, t1 = pl.token_range(l)
+        out.append(np.ascontiguousarray(X[g * pl.Bl:(g + 1) * pl.Bl, t0:t1]))
+    return out
+
+
+def gather_uneven(shards: list, pl: Plan) -> np.ndarray:
+    """Inverse of :func:`partition_uneven`."""
+    H, D = shards[0].shape[2:]
+    out = np.empty((pl.B, pl.S, H, D), dtype=shards[0].dtype)
+    for r in range(pl.N):
+        g, l = divmod(r, pl.K)
+        t0, t1 = pl.token_range(l)
+        assert shards[r].shape == (pl.Bl, t1 - t0, H, D)
+        out[g * pl.Bl:(g + 1) * pl.Bl, t0:t1] = shards[r]
+    return out
+
+
+def s2h_uneven(shards: list, pl: Plan) -> np.ndarray:
+    """First all-to-all from uneven shards: head[gK+m][bl][s][h'] = seq[gK+src][bl][s - src T][m H/K + h'] with src
+    the rank whose token range holds s.  A tensor with fewer heads than the group has ranks is replicated as in
+    :func:`s2h_replicated` (local rank m receives head m // (K/H))."""
+    H, D = shards[0].shape[2:]
+    K = pl.K
+    assert H % K == 0 or K % H == 0
+    Hl, rep = (H // K, 1) if H % K == 0 else (1, K // H)
+    out = np.empty((pl.N, pl.Bl, pl.S, Hl, D), dtype=shards[0].dtype)
+    for g in range(pl.G):
+        for m in range(K):
+            h0 = m * Hl if rep == 1 else m // rep
+            for src in range(K):
+                t0, t1 = pl.token_range(src)
+                out[g * K + m, :, t0:t1] = shards[g * K + src][:, :, h0:h0 + Hl, :]
+    return out
+
+
+def h2s_uneven(head: np.ndarray, pl: Plan, H: int | None = None) -> list:
+    """Reverse all-to-all to uneven shards.  With H given and smaller than K the tensor is the gradient of a replicated
+    K/V tensor and the copies are summed as in :func:`h2s_sum_replicated`."""
+    N, Bl, S, Hl, D = head.shape
+    K = pl.K
+    assert (N, Bl, S) == (pl.N, pl.Bl, pl.S)
+    if H is None:
+        H = Hl * K
+    rep = 1 if H % K == 0 else K // H
+    out = []
+    for r in range(N):
+        g, dst = divmod(r, K)
+        t0, t1 = pl.token_range(dst)
+        o = np.zeros((Bl, t1 - t0, H, D), dtype=head.dtype)
+        for m in range(K):
+            if rep == 1:
+                o[:, :, m * Hl:(m + 1) * Hl, :] = head[g * K + m, :, t0:t1]
+            else:
+                o[:, :, m // rep, :] += head[g * K + m, :, t0:t1, 0, :]
+        out.append(o)
     return out
 
 
@@ -257,9 +347,12 @@ def layer_bwd(Xq, Xk, Xv, XdO, pl: Plan, scale: float | None = None, causal: boo
     collect.  Returns dict with head- and sequence-sharded gradients and the global ones."""
     Hkv = Xk.shape[2]
     replicated = Hkv % pl.K != 0                  # more ranks in a group than KV heads
-    kv_s2h = s2h_replicated if replicated else s2h
-    qh, doh = s2h(partition(Xq, pl), pl), s2h(partition(XdO, pl), pl)
-    kh, vh = kv_s2h(partition(Xk, pl), pl), kv_s2h(partition(Xv, pl), pl)
+    if pl.uneven:
+        qh, doh, kh, vh = (s2h_uneven(partition_uneven(X, pl), pl) for X in (Xq, XdO, Xk, Xv))
+    else:
+        kv_s2h = s2h_replicated if replicated else s2h
+        qh, doh = s2h(partition(Xq, pl), pl), s2h(partition(XdO, pl), pl)
+        kh, vh = kv_s2h(partition(Xk, pl), pl), kv_s2h(partition(Xv, pl), pl)
     dqh = np.empty(qh.shape, dtype=np.float64)
     dkh = np.empty(kh.shape, dtype=np.float64)
     dvh = np.empty(kh.shape, dtype=np.float64)
@@ -268,6 +361,10 @@ def layer_bwd(Xq, Xk, Xv, XdO, pl: Plan, scale: float | None = None, causal: boo
         dqh[r], dkh[r], dvh[r] = g["dQ"], g["dK"], g["dV"]
     out = dict(dq_head=dqh, dk_head=dkh, dv_head=dvh, do_head=doh)
     for n, a in (("dq", dqh), ("dk", dkh), ("dv", dvh)):
+        if pl.uneven:
+            out[n + "_seq"] = h2s_uneven(a, pl, None if n == "dq" else Hkv)
+            out[n + "_global"] = gather_uneven(out[n + "_seq"], pl)
+            continue
         out[n + "_seq"] = h2s_sum_replicated(a, pl, Hkv) if (replicated and n != "dq") else h2s(a, pl)
         out[n + "_global"] = gather(out[n + "_seq"], pl)
     return out
@@ -282,17 +379,22 @@ def layer_fwd(Xq: np.ndarray, Xk: np.ndarray, Xv: np.ndarray, pl: Plan,
 
     Xq [B,S,Hq,D], Xk,Xv [B,S,Hkv,D] uint16.  Returns a dict with every intermediate
     (seq shards, head shards, per-rank O/LSE in fp64) and the global O [B,S,Hq,D]."""
-    qs, ks, vs = partition(Xq, pl), partition(Xk, pl), partition(Xv, pl)
-    kv_s2h = s2h if Xk.shape[2] % pl.K == 0 else s2h_replicated
-    qh, kh, vh = s2h(qs, pl), kv_s2h(ks, pl), kv_s2h(vs, pl)
+    if pl.uneven:
+        qs, ks, vs = (partition_uneven(X, pl) for X in (Xq, Xk, Xv))
+        qh, kh, vh = (s2h_uneven(x, pl) for x in (qs, ks, vs))
+    else:
+        qs, ks, vs = partition(Xq, pl), partition(Xk, pl), partition(Xv, pl)
+        kv_s2h = s2h if Xk.shape[2] % pl.K == 0 else s2h_replicated
+        qh, kh, vh = s2h(qs, pl), kv_s2h(ks, pl), kv_s2h(vs, pl)
     N = pl.N
     oh = np.empty(qh.shape, dtype=np.float64)
     lse = np.empty((N, pl.Bl, qh.shape[3], pl.S), dtype=np.float64)
     for r in range(N):
         oh[r], lse[r] = attn_fwd(qh[r], kh[r], vh[r], scale, causal)
-    os_ = h2s(oh, pl)
+    os_ = h2s_uneven(oh, pl) if pl.uneven else h2s(oh, pl)
     return dict(q_seq=qs, k_seq=ks, v_seq=vs, q_head=qh, k_head=kh, v_head=vh,
-                o_head=oh, lse_head=lse, o_seq=os_, o_global=gather(os_, pl))
+                o_head=oh, lse_head=lse, o_seq=os_,
+                o_global=gather_uneven(os_, pl) if pl.uneven else gather(os_, pl))
 
 
 # ------------------------------------------------------------------- projections
