@@ -13,10 +13,11 @@
  *
  * Notation: N ranks; B micro-batch (sequences); G groups (G = B is BASP, G = 1 standard
  * Ulysses); K = N/G ranks per group; Bl = B/G sequences per group; S tokens per sequence;
- * T = S/K tokens per rank and sequence; Hq / Hkv query / key-value heads; D head dim.
+ * T = ceil(S/K) tokens per rank and sequence; Hq / Hkv query / key-value heads; D head dim.
  *
  * Shard layouts (dense, row-major, bf16 unless stated):
- *   sequence-sharded  rank r holds [Bl][T][H][D]    (tokens l*T..(l+1)*T of its sequences)
+ *   sequence-sharded  rank r holds [Bl][T][H][D]    (tokens l*T..(l+1)*T of its sequences; where K does not divide S
+ *                     the last rank of a group holds [Bl][S-(K-1)*T][H][D], see basp_plan_create)
  *   head-sharded      rank r holds [Bl][S][H/K][D]  (heads l*H/K..(l+1)*H/K, all tokens)
  *   LSE               rank r holds fp32 [Bl][Hq/K][S] (natural log of the softmax denominator)
  * with l = r mod K the local rank and g = r / K the group.
@@ -73,10 +74,12 @@ typedef struct basp_plan_info {
     int group_size;        /* K = N / G  (all-to-all participants; Table I)               */
     int num_groups;        /* G                                                           */
     int seqs_per_group;    /* Bl = B / G                                                  */
-    int tokens_per_rank;   /* T = S / K  (per sequence; tokens per rank = Bl * T = B*S/N) */
+    int tokens_per_rank;   /* T = ceil(S / K)  (per sequence; tokens per rank = Bl * T = B*S/N when K | S) */
+    int tokens_last_rank;  /* tokens per sequence of a group's LAST rank: T, or S - (K-1)*T when K does not divide S */
     int q_heads_per_rank;  /* Hq / K                                                      */
     int kv_heads_per_rank; /* Hkv / K                                                     */
-    size_t q_shard_elems;  /* elements of one rank's Q (or O) shard, either layout        */
+    size_t q_shard_elems;  /* elements of one rank's Q (or O) shard, either layout (a short last rank's */
+                           /* sequence-sharded shard holds tokens_last_rank instead of T tokens)   */
     size_t kv_shard_elems; /* elements of one rank's K (or V) shard (sequence-sharded;    */
                            /* head-sharded too unless KV heads are replicated, see below)  */
     size_t lse_shard_elems;/* fp32 elements of one rank's LSE                             */
@@ -95,7 +98,7 @@ typedef struct basp_rank_info {
  * Algorithm 2 (group = r / K, local = r mod K, chunk = S / K), generalised to G groups
  * as in the workload-equivalence paragraph of Section IV-C.
  * Errors: BASP_ERR_NULL; BASP_ERR_INVALID for N mod G != 0, B mod G != 0, B > N in BASP
- * mode (the paper's data-parallel fallback is not provided), S mod K != 0, Hq mod Hkv != 0,
+ * mode (the paper's data-parallel fallback is not provided), an empty last rank (below), Hq mod Hkv != 0,
  * Hq mod K != 0, or Hkv and K with neither Hkv mod K = 0 nor K mod Hkv = 0; BASP_ERR_UNSUPPORTED for
  * dtype != bf16, N > BASP_MAX_RANKS or a head slice whose row ((H/K)*D*2 bytes) is not a multiple of 16 bytes.
  * A group with MORE ranks than KV heads (K mod Hkv = 0, K > Hkv; the paper does not treat grouped-query attention)
@@ -104,6 +107,10 @@ typedef struct basp_rank_info {
  * [Bl][S][1][D], larger than the sequence-sharded one.  On the way back such a tensor carries gradients:
  * basp_reshard_h2s (and basp_reshard_grads_h2s for dK, dV) ADDS the K/Hkv copies of a head (fp32 sum, one rounding),
  * which is what the backward pass needs; basp_reshard_h2s is therefore not the inverse of basp_reshard_s2h for it.
+ * A sequence length that K does not divide (Algorithm 2 writes the chunk as L / K and the paper says nothing about a
+ * remainder): the chunk is T = ceil(S / K); local rank l holds tokens [l*T, min((l+1)*T, S)), so only the last rank of
+ * a group is short, and its SEQUENCE-sharded shards are the compact [Bl][S - (K-1)*T][H][D] (head-sharded shards and LSE
+ * do not change: every rank holds whole sequences there).  (K-1)*T >= S, an empty last rank, is BASP_ERR_INVALID.
  * On success *out owns a host object; release it with basp_plan_destroy. */
 int basp_plan_create(const basp_config *cfg, basp_plan **out);
 int basp_plan_destroy(basp_plan *plan);

@@ -42,7 +42,7 @@ class basp_config(Structure):
 
 class basp_plan_info(Structure):
     _fields_ = [(n, c_int) for n in ("group_size", "num_groups", "seqs_per_group", "tokens_per_rank",
-                                     "q_heads_per_rank", "kv_heads_per_rank")] + \
+                                     "tokens_last_rank", "q_heads_per_rank", "kv_heads_per_rank")] + \
                [(n, c_size_t) for n in ("q_shard_elems", "kv_shard_elems", "lse_shard_elems")]
 
 
@@ -136,6 +136,12 @@ class Plan:
         self.K, self.G, self.Bl, self.T = info.group_size, info.num_groups, info.seqs_per_group, info.tokens_per_rank
         self.S, self.Hq, self.Hkv, self.D = cfg.seq_len, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
         self.Hq_l, self.Hkv_l = info.q_heads_per_rank, info.kv_heads_per_rank
+        self.T_last = info.tokens_last_rank
+
+    def rank_tokens(self, r: int) -> int:
+        """Tokens per sequence in rank r's sequence-sharded shards (the last rank of a group is short when the group
+        size does not divide the sequence length)."""
+        return self.T_last if r % self.K == self.K - 1 else self.T
 
     def __del__(self, _destroy=lib.basp_plan_destroy):
         h, self.handle = getattr(self, "handle", None), None

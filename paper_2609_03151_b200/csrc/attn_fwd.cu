@@ -4,7 +4,8 @@
 //
 // The same kernel serves two addressings of its operands:
 //   head-sharded  rank r holds [Bl][S][H/K][D]; tile (bl, s0, h) is rows bl*S+s0.. of rank r
-//   fused         operands stay SEQUENCE-sharded [Bl][T][H][D]; the tile at sequence position
+//   fused         operands stay SEQUENCE-sharded [Bl][T][H][D] (T a multiple of the tile; the last rank of a group may
+//                 hold fewer tokens); the tile at sequence position
 //                 s0 of local head h lives on rank gK + s0/T, rows bl*T + s0 mod T, head l*H/K+h
 //                 (the all-to-all of Section IV-C folded into the tile fetch / the O store).
 #include <cuda.h>
@@ -36,13 +37,13 @@ template <int R>
 int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const *k, const void *const *v,
                     void *const *o, float *const *lse, float scale, bool fused, const int range[4], cudaStream_t st) {
     AttnParams<R> prm;
-    const uint64_t rows = (uint64_t)pl->Bl * (fused ? pl->T : pl->S);
     const int hq = fused ? pl->Hq : pl->Hq_l, hkv = fused ? pl->Hkv : pl->Hkv_l;
     // Operands of ranks outside the launch's range are not touched: with head-sharded operands only the ranks of the
     // range, with sequence-sharded (fused) operands every member of their groups.
     const int need_lo = fused ? range[0] / pl->K * pl->K : range[0];
     const int need_hi = fused ? (range[0] + range[1] + pl->K - 1) / pl->K * pl->K : range[0] + range[1];
     for (int r = need_lo; r < need_hi; ++r) {
+        const uint64_t rows = (uint64_t)pl->Bl * (fused ? basp_rank_tokens(pl, r % pl->K) : pl->S);
         int rc = tmap::encode_rows_heads_d(&prm.q[r], q[r], rows, hq, pl->D, kTile);
         if (rc == BASP_OK) rc = tmap::encode_rows_heads_d(&prm.k[r], k[r], rows, hkv, pl->D, kTile);
         if (rc == BASP_OK) rc = tmap::encode_rows_heads_d(&prm.v[r], v[r], rows, hkv, pl->D, kTile);
@@ -50,7 +51,7 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
         prm.o[r] = (__nv_bfloat16 *)o[r];
         prm.lse[r] = lse ? lse[r] : nullptr;
     }
-    prm.n_ranks = pl->N; prm.K = pl->K; prm.Bl = pl->Bl; prm.S = pl->S; prm.T = pl->T;
+    prm.n_ranks = pl->N; prm.K = pl->K; prm.Bl = pl->Bl; prm.S = pl->S; prm.T = pl->T; prm.T_last = pl->T_last;
     prm.Hq_l = pl->Hq_l; prm.Hkv_l = pl->Hkv_l; prm.q_per_kv = pl->Hq_l / pl->Hkv_l;
     prm.kv_rep = pl->kv_rep;
     prm.o_heads = hq;

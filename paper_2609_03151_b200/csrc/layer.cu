@@ -13,16 +13,21 @@ int basp_attn_dispatch_range(const basp_plan *pl, const void *const *q, const vo
 namespace {
 size_t q_shard_bytes(const basp_plan *p) { return (size_t)p->Bl * p->T * p->Hq * p->D * 2; }
 size_t kv_shard_bytes(const basp_plan *p) { return (size_t)p->Bl * p->T * p->Hkv * p->D * 2; }
+// head-sharded Q (or O) of one rank: the same bytes as a sequence-sharded shard when K divides S
+size_t q_head_bytes(const basp_plan *p) { return (size_t)p->Bl * p->S * p->Hq_l * p->D * 2; }
 // head-sharded K or V of one rank: the same bytes unless KV heads are replicated inside the group
 size_t kv_head_bytes(const basp_plan *p) { return (size_t)p->Bl * p->S * p->Hkv_l * p->D * 2; }
 }  // namespace
 
 extern "C" size_t basp_workspace_bytes(const basp_plan *p) {
     if (!p) return 0;
-    return (size_t)p->N * (2 * q_shard_bytes(p) + 2 * kv_head_bytes(p));   // head-sharded Q, K, V, O
+    return (size_t)p->N * (2 * q_head_bytes(p) + 2 * kv_head_bytes(p));   // head-sharded Q, K, V, O
 }
 
-extern "C" size_t basp_host_arena_bytes(const basp_plan *p) { return basp_workspace_bytes(p); }
+extern "C" size_t basp_host_arena_bytes(const basp_plan *p) {
+    if (!p) return 0;
+    return (size_t)p->N * (2 * q_shard_bytes(p) + 2 * kv_shard_bytes(p));  // sequence-sharded Q, K, V, O
+}
 
 extern "C" int basp_layer_fwd(const basp_plan *p, const void *const *q_seq, const void *const *k_seq,
                               const void *const *v_seq, void *const *o_seq, float *const *lse_shards,
@@ -32,7 +37,7 @@ extern "C" int basp_layer_fwd(const basp_plan *p, const void *const *q_seq, cons
     if (workspace_bytes < basp_workspace_bytes(p)) return BASP_ERR_WORKSPACE;
     char *w = (char *)workspace;
     void *qh[BASP_MAX_RANKS], *kh[BASP_MAX_RANKS], *vh[BASP_MAX_RANKS], *oh[BASP_MAX_RANKS];
-    const size_t qb = q_shard_bytes(p), kb = kv_head_bytes(p);
+    const size_t qb = q_head_bytes(p), kb = kv_head_bytes(p);
     for (int r = 0; r < p->N; ++r) {
         qh[r] = w + (size_t)r * qb;
         kh[r] = w + (size_t)p->N * qb + (size_t)r * kb;
@@ -50,7 +55,7 @@ extern "C" int basp_layer_workspace_shards(const basp_plan *p, void *workspace, 
                                            void **v_head, void **o_head) {
     if (!p || !workspace || !q_head || !k_head || !v_head || !o_head) return BASP_ERR_NULL;
     char *w = (char *)workspace;
-    const size_t qb = q_shard_bytes(p), kb = kv_head_bytes(p);
+    const size_t qb = q_head_bytes(p), kb = kv_head_bytes(p);
     for (int r = 0; r < p->N; ++r) {
         q_head[r] = w + (size_t)r * qb;
         k_head[r] = w + (size_t)p->N * qb + (size_t)r * kb;
@@ -63,7 +68,7 @@ extern "C" int basp_layer_workspace_shards(const basp_plan *p, void *workspace, 
 extern "C" size_t basp_layer_bwd_workspace_bytes(const basp_plan *p) {
     if (!p) return 0;
     // head-sharded dO and dQ (query-sized), dK and dV (key-sized), then the attention-backward workspace
-    return (size_t)p->N * (2 * q_shard_bytes(p) + 2 * kv_head_bytes(p)) + basp_attn_bwd_workspace_bytes(p);
+    return (size_t)p->N * (2 * q_head_bytes(p) + 2 * kv_head_bytes(p)) + basp_attn_bwd_workspace_bytes(p);
 }
 
 extern "C" int basp_layer_bwd(const basp_plan *p, const void *const *q_head, const void *const *k_head,
@@ -76,7 +81,7 @@ extern "C" int basp_layer_bwd(const basp_plan *p, const void *const *q_head, con
     if (workspace_bytes < basp_layer_bwd_workspace_bytes(p)) return BASP_ERR_WORKSPACE;
     char *w = (char *)workspace;
     void *doh[BASP_MAX_RANKS], *dqh[BASP_MAX_RANKS], *dkh[BASP_MAX_RANKS], *dvh[BASP_MAX_RANKS];
-    const size_t qb = q_shard_bytes(p), kb = kv_head_bytes(p);
+    const size_t qb = q_head_bytes(p), kb = kv_head_bytes(p);
     for (int r = 0; r < p->N; ++r) {
         doh[r] = w + (size_t)r * qb;
         dqh[r] = w + (size_t)p->N * qb + (size_t)r * qb;
@@ -95,7 +100,7 @@ extern "C" int basp_layer_bwd(const basp_plan *p, const void *const *q_head, con
 extern "C" size_t basp_layer_bwd_seq_workspace_bytes(const basp_plan *p) {
     if (!p) return 0;
     // head-sharded Q, O, dO, dQ (query-sized), K, V, dK, dV (key-sized), then the attention-backward workspace
-    return (size_t)p->N * (4 * q_shard_bytes(p) + 4 * kv_head_bytes(p)) + basp_attn_bwd_workspace_bytes(p);
+    return (size_t)p->N * (4 * q_head_bytes(p) + 4 * kv_head_bytes(p)) + basp_attn_bwd_workspace_bytes(p);
 }
 
 extern "C" int basp_layer_bwd_seq(const basp_plan *p, const void *const *q_seq, const void *const *k_seq,
@@ -109,7 +114,7 @@ extern "C" int basp_layer_bwd_seq(const basp_plan *p, const void *const *q_seq, 
     char *w = (char *)workspace;
     void *qh[BASP_MAX_RANKS], *kh[BASP_MAX_RANKS], *vh[BASP_MAX_RANKS], *oh[BASP_MAX_RANKS], *doh[BASP_MAX_RANKS],
         *dqh[BASP_MAX_RANKS], *dkh[BASP_MAX_RANKS], *dvh[BASP_MAX_RANKS];
-    const size_t qb = q_shard_bytes(p), kb = kv_head_bytes(p);
+    const size_t qb = q_head_bytes(p), kb = kv_head_bytes(p);
     const size_t n = (size_t)p->N;
     for (int r = 0; r < p->N; ++r) {
         qh[r] = w + (size_t)r * qb;
@@ -194,6 +199,9 @@ extern "C" int basp_layer_fwd_host(const basp_plan *p, const void *const *q_seq_
         od[r] = w + (size_t)p->N * (qb + 2 * kb) + (size_t)r * qb;
     }
     const bool by_chunk = p->causal && p->T % 256 == 0;     // a launch per local rank's rows, else per group
+    // bytes of rank r's shards (the last rank of a group is short when K does not divide S)
+    auto qbytes = [&](int r) { return qb / p->T * basp_rank_tokens(p, r % p->K); };
+    auto kbytes = [&](int r) { return kb / p->T * basp_rank_tokens(p, r % p->K); };
     BASP_CUDA_TRY(cudaEventRecord(pipe->start, st));
     BASP_CUDA_TRY(cudaStreamWaitEvent(pipe->in, pipe->start, 0));
     BASP_CUDA_TRY(cudaStreamWaitEvent(pipe->out, pipe->start, 0));
@@ -206,44 +214,44 @@ extern "C" int basp_layer_fwd_host(const basp_plan *p, const void *const *q_seq_
                 const int r0 = g * p->K;
                 if (l == p->K - 1) {
                     for (int j = 0; j < p->K; ++j) {
-                        BASP_CUDA_TRY(cudaMemcpyAsync(kd[r0 + j], k_seq_host[r0 + j], kb, cudaMemcpyHostToDevice, pipe->in));
-                        BASP_CUDA_TRY(cudaMemcpyAsync(vd[r0 + j], v_seq_host[r0 + j], kb, cudaMemcpyHostToDevice, pipe->in));
+                        BASP_CUDA_TRY(cudaMemcpyAsync(kd[r0 + j], k_seq_host[r0 + j], kbytes(r0 + j), cudaMemcpyHostToDevice, pipe->in));
+                        BASP_CUDA_TRY(cudaMemcpyAsync(vd[r0 + j], v_seq_host[r0 + j], kbytes(r0 + j), cudaMemcpyHostToDevice, pipe->in));
                     }
                 }
-                BASP_CUDA_TRY(cudaMemcpyAsync(qd[r0 + l], q_seq_host[r0 + l], qb, cudaMemcpyHostToDevice, pipe->in));
+                BASP_CUDA_TRY(cudaMemcpyAsync(qd[r0 + l], q_seq_host[r0 + l], qbytes(r0 + l), cudaMemcpyHostToDevice, pipe->in));
                 BASP_CUDA_TRY(cudaEventRecord(pipe->arrived[r0 + l], pipe->in));
             }
         for (int l = p->K - 1; l >= 0; --l)
             for (int g = 0; g < p->G; ++g) {
                 const int r0 = g * p->K;
                 BASP_CUDA_TRY(cudaStreamWaitEvent(st, pipe->arrived[r0 + l], 0));   // implies the group's K and V
-                const int range[4] = {r0, p->K, l * (p->T / 256), p->T / 256};
+                const int range[4] = {r0, p->K, l * (p->T / 256), (basp_rank_tokens(p, l) + 255) / 256};
                 rc = basp_attn_dispatch_range(p, qd, kd, vd, od, nullptr, softmax_scale, true, range, stream);
                 if (rc != BASP_OK) return rc;
                 BASP_CUDA_TRY(cudaEventRecord(pipe->computed[r0 + l], st));
                 BASP_CUDA_TRY(cudaStreamWaitEvent(pipe->out, pipe->computed[r0 + l], 0));
-                BASP_CUDA_TRY(cudaMemcpyAsync(o_seq_host[r0 + l], od[r0 + l], qb, cudaMemcpyDeviceToHost, pipe->out));
+                BASP_CUDA_TRY(cudaMemcpyAsync(o_seq_host[r0 + l], od[r0 + l], qbytes(r0 + l), cudaMemcpyDeviceToHost, pipe->out));
             }
     } else {
         for (int g = 0; g < p->G; ++g) {
             const int r0 = g * p->K;
             for (int l = 0; l < p->K; ++l) {
-                BASP_CUDA_TRY(cudaMemcpyAsync(kd[r0 + l], k_seq_host[r0 + l], kb, cudaMemcpyHostToDevice, pipe->in));
-                BASP_CUDA_TRY(cudaMemcpyAsync(vd[r0 + l], v_seq_host[r0 + l], kb, cudaMemcpyHostToDevice, pipe->in));
-                BASP_CUDA_TRY(cudaMemcpyAsync(qd[r0 + l], q_seq_host[r0 + l], qb, cudaMemcpyHostToDevice, pipe->in));
+                BASP_CUDA_TRY(cudaMemcpyAsync(kd[r0 + l], k_seq_host[r0 + l], kbytes(r0 + l), cudaMemcpyHostToDevice, pipe->in));
+                BASP_CUDA_TRY(cudaMemcpyAsync(vd[r0 + l], v_seq_host[r0 + l], kbytes(r0 + l), cudaMemcpyHostToDevice, pipe->in));
+                BASP_CUDA_TRY(cudaMemcpyAsync(qd[r0 + l], q_seq_host[r0 + l], qbytes(r0 + l), cudaMemcpyHostToDevice, pipe->in));
             }
             BASP_CUDA_TRY(cudaEventRecord(pipe->arrived[r0], pipe->in));
         }
         for (int g = 0; g < p->G; ++g) {
             const int r0 = g * p->K;
             BASP_CUDA_TRY(cudaStreamWaitEvent(st, pipe->arrived[r0], 0));
-            const int range[4] = {r0, p->K, 0, (p->S / 128 + 1) / 2};
+            const int range[4] = {r0, p->K, 0, ((p->S + 127) / 128 + 1) / 2};
             rc = basp_attn_dispatch_range(p, qd, kd, vd, od, nullptr, softmax_scale, true, range, stream);
             if (rc != BASP_OK) return rc;
             BASP_CUDA_TRY(cudaEventRecord(pipe->computed[r0], st));
             BASP_CUDA_TRY(cudaStreamWaitEvent(pipe->out, pipe->computed[r0], 0));
             for (int l = 0; l < p->K; ++l)
-                BASP_CUDA_TRY(cudaMemcpyAsync(o_seq_host[r0 + l], od[r0 + l], qb, cudaMemcpyDeviceToHost, pipe->out));
+                BASP_CUDA_TRY(cudaMemcpyAsync(o_seq_host[r0 + l], od[r0 + l], qbytes(r0 + l), cudaMemcpyDeviceToHost, pipe->out));
         }
     }
     BASP_CUDA_TRY(cudaEventRecord(pipe->done, pipe->out));

@@ -16,7 +16,10 @@ extern "C" int basp_plan_create(const basp_config *cfg, basp_plan **out) {
     if (G == B && B > N) return BASP_ERR_INVALID;               // data-parallel fallback: not a plan
     if (N % G != 0 || B % G != 0) return BASP_ERR_INVALID;      // Algorithm 1: assert N mod B = 0
     const int K = N / G;                                         // Algorithm 1: K = N / B
-    if (S % K != 0) return BASP_ERR_INVALID;                     // Algorithm 2: chunk = L / K
+    // Algorithm 2: chunk = L / K.  Where K does not divide L (the paper is silent) the chunk is rounded up and the
+    // group's last rank holds the short remainder, which must not be empty.
+    const int T = (S + K - 1) / K, T_last = S - (K - 1) * T;
+    if (T_last <= 0) return BASP_ERR_INVALID;
     // Each rank takes Hq/K query heads and their KV heads.  A group with more ranks than KV heads replicates: KV head
     // h goes to the K/Hkv consecutive local ranks whose query heads read it (one KV head per rank).
     if (Hq % Hkv != 0 || Hq % K != 0) return BASP_ERR_INVALID;
@@ -29,7 +32,7 @@ extern "C" int basp_plan_create(const basp_config *cfg, basp_plan **out) {
     basp_plan *p = new (std::nothrow) basp_plan;
     if (!p) return BASP_ERR_INVALID;
     p->cfg = *cfg;
-    p->N = N; p->B = B; p->G = G; p->K = K; p->Bl = B / G; p->S = S; p->T = S / K;
+    p->N = N; p->B = B; p->G = G; p->K = K; p->Bl = B / G; p->S = S; p->T = T; p->T_last = T_last;
     p->Hq = Hq; p->Hkv = Hkv; p->D = D; p->Hq_l = Hq / K; p->Hkv_l = Hkv_l; p->kv_rep = kv_rep;
     p->causal = cfg->causal;
     *out = p;
@@ -48,6 +51,7 @@ extern "C" int basp_plan_get_info(const basp_plan *p, basp_plan_info *info) {
     info->num_groups = p->G;
     info->seqs_per_group = p->Bl;
     info->tokens_per_rank = p->T;
+    info->tokens_last_rank = p->T_last;
     info->q_heads_per_rank = p->Hq_l;
     info->kv_heads_per_rank = p->Hkv_l;
     // Workload equivalence (Section IV-C): Bl*T*H*D = (B*S/N)*H*D for every grouping.
@@ -66,7 +70,7 @@ extern "C" int basp_plan_get_rank(const basp_plan *p, int r, basp_rank_info *inf
     info->seq_begin = g * p->Bl;                // Algorithm 2: seq_start = my_group (Bl = 1)
     info->seq_end = (g + 1) * p->Bl;
     info->token_begin = l * p->T;               // Algorithm 2: token_start = local * chunk
-    info->token_end = (l + 1) * p->T;
+    info->token_end = l * p->T + basp_rank_tokens(p, l);
     info->q_head_begin = l * p->Hq_l;
     info->q_head_end = (l + 1) * p->Hq_l;
     info->kv_head_begin = p->kv_rep > 1 ? l / p->kv_rep : l * p->Hkv_l;

@@ -33,6 +33,7 @@ struct GemmParams {
     CUtensorMap a[R];
     CUtensorMap w;
     int n_ranks, M, N, K;
+    int M_last;                            // rows of the last rank of a group (= M unless the group size does not divide S)
     int n_seg;
     int seg_begin[3], seg_ld[3];           // first output column of the segment; row pitch of its tensor (elements)
     __nv_bfloat16 *seg_ptr[3][R];
@@ -41,6 +42,7 @@ struct GemmParams {
     // 32 consecutive positions, so a warp's read of one feature is one 128-byte line), position of a row = the token's
     // place in its sequence: local rank (r mod rope_K) * rope_T + row mod rope_T
     int rope_segs, rope_half, rope_T, rope_K, rope_S;
+    int rope_T_last;                       // tokens per sequence of a group's last rank
     const float *rope_cos, *rope_sin;
     int *status;
 };
@@ -138,6 +140,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) proj_gemm_kernel(const __grid
             int seg = 0;
             while (seg + 1 < p.n_seg && n * kBN >= p.seg_begin[seg + 1]) ++seg;
             const int grow = m * kBM + row;
+            const bool short_rank = r % p.rope_K == p.rope_K - 1;
+            const int Mr = short_rank ? p.M_last : p.M;
             __nv_bfloat16 *dst = p.seg_ptr[seg][r] + (size_t)grow * p.seg_ld[seg] + (n * kBN - p.seg_begin[seg]);
             GEMM_WAIT(&bars.acc_full[acc], (tile_cnt >> 1) & 1, 3, tile);
             tc_fence_after();
@@ -147,7 +151,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) proj_gemm_kernel(const __grid
                 // on the fp32 accumulators, one rounding to bf16 afterwards.  A thread owns a row, so both halves of every
                 // head of the tile are in its own TMEM lane.
                 const int half = p.rope_half, D2 = 2 * half;
-                const int pos = (r % p.rope_K) * p.rope_T + (grow % p.rope_T);
+                const int pos = (r % p.rope_K) * p.rope_T + (grow % (short_rank ? p.rope_T_last : p.rope_T));
                 const float *ct = p.rope_cos + pos, *sn = p.rope_sin + pos;
                 for (int j0 = 0; j0 < half; j0 += 32) {
                     // the angles depend on (position, feature) only: one fetch of 32 features serves every head of the tile
@@ -168,7 +172,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) proj_gemm_kernel(const __grid
                             __syncwarp();
                             if (lane == 0) mbar_arrive(&bars.acc_empty[acc]);
                         }
-                        if (grow < p.M) {
+                        if (grow < Mr) {
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 float yl[8], yh[8];
@@ -201,7 +205,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) proj_gemm_kernel(const __grid
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars.acc_empty[acc]);
                 }
-                if (grow < p.M) {
+                if (grow < Mr) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         uint4 o4;
@@ -244,12 +248,12 @@ int gemm_launch(const basp_plan *pl, const void *const *a, const void *w, int M,
                 int n_seg, const Rope &rope, cudaStream_t st) {
     GemmParams<R> prm;
     for (int r = 0; r < pl->N; ++r) {
-        int rc = tmap::encode_rows_heads_d(&prm.a[r], a[r], (uint64_t)M, 1, (uint64_t)K, kBM);
+        int rc = tmap::encode_rows_heads_d(&prm.a[r], a[r], (uint64_t)pl->Bl * basp_rank_tokens(pl, r % pl->K), 1, (uint64_t)K, kBM);
         if (rc != BASP_OK) return rc;
     }
     int rc = tmap::encode_rows_heads_d(&prm.w, w, (uint64_t)N, 1, (uint64_t)K, kBN);
     if (rc != BASP_OK) return rc;
-    prm.n_ranks = pl->N; prm.M = M; prm.N = N; prm.K = K; prm.n_seg = n_seg;
+    prm.n_ranks = pl->N; prm.M = M; prm.M_last = pl->Bl * pl->T_last; prm.N = N; prm.K = K; prm.n_seg = n_seg;
     int col = 0;
     for (int s = 0; s < n_seg; ++s) {
         prm.seg_begin[s] = col;
@@ -257,7 +261,7 @@ int gemm_launch(const basp_plan *pl, const void *const *a, const void *w, int M,
         for (int r = 0; r < pl->N; ++r) prm.seg_ptr[s][r] = (__nv_bfloat16 *)segs[s].ptrs[r];
         col += segs[s].cols;
     }
-    prm.rope_segs = rope.segs; prm.rope_half = pl->D / 2; prm.rope_T = pl->T; prm.rope_K = pl->K; prm.rope_S = pl->S;
+    prm.rope_segs = rope.segs; prm.rope_half = pl->D / 2; prm.rope_T = pl->T; prm.rope_T_last = pl->T_last; prm.rope_K = pl->K; prm.rope_S = pl->S;
     prm.rope_cos = rope.cos; prm.rope_sin = rope.sin;
     prm.status = basp_status_device_ptr();
     if (!prm.status) return BASP_ERR_CUDA;

@@ -3,6 +3,7 @@
 //
 //   s2h: head[gK+m][bl][s][h'][d] = seq[gK + s/T][bl][s mod T][m*H/K + h'][d]
 //   h2s: the inverse map.
+// (T = ceil(S/K); where K does not divide S the last rank of a group holds the short remainder, a compact shard.)
 //
 // The unit moved is a 16-byte vector.  Walking the SEQUENCE-sharded side in memory order, a
 // token row of H*D elements is K consecutive runs of (H/K)*D elements, run m belonging to
@@ -28,7 +29,7 @@ struct ReshardTensor {
     uint32_t row_v;            // vectors per token row on the sequence-sharded side (K runs)
     uint32_t run_v;            // vectors per run = (H/K)*D*2/16 (one head when replicated)
     uint32_t rep;              // head-side ranks that receive each run (1; K/H when a group has more ranks than heads)
-    uint32_t shard_v;          // vectors per rank shard
+    uint32_t shard_v;          // vectors per rank shard (of T tokens; a short last rank has fewer)
     uint32_t chunks_per_shard;
     uint32_t chunk_begin;      // first CTA index of this tensor
     FastDiv div_row, div_run;
@@ -37,8 +38,9 @@ struct ReshardTensor {
 struct ReshardParams {
     int n_tensors;
     uint32_t r_begin, r_count; // sequence-side ranks this launch walks
-    uint32_t K, T, S;
-    FastDiv div_T;
+    uint32_t K, T, S, Bl;
+    uint32_t T_last;           // tokens per sequence of a group's last rank (= T when K divides S)
+    FastDiv div_T, div_T_last;
     ReshardTensor t[3];
 };
 
@@ -67,6 +69,10 @@ __global__ void __launch_bounds__(kThreads) reshard_kernel(const __grid_constant
     const uint32_t r = p.r_begin + ri;
     const uint32_t g = r / p.K, l = r - g * p.K;
     const uint32_t v0 = chunk * kChunkV + threadIdx.x;
+    const bool last = l == p.K - 1;
+    const uint32_t Tr = last ? p.T_last : p.T;                       // this rank's tokens per sequence
+    const FastDiv div_Tr = last ? p.div_T_last : p.div_T;
+    const uint32_t shard_v = last ? p.Bl * Tr * t.row_v : t.shard_v;
 
     const uint4 *seq = reinterpret_cast<const uint4 *>(t.seq[r]);
     const uint4 *hp[kUnroll];   // address on the head-sharded side of each vector (of its first copy when replicated)
@@ -74,13 +80,13 @@ __global__ void __launch_bounds__(kThreads) reshard_kernel(const __grid_constant
 #pragma unroll
     for (int i = 0; i < kUnroll; ++i) {
         const uint32_t v = v0 + i * kThreads;
-        const uint32_t vv = v < t.shard_v ? v : 0;
+        const uint32_t vv = v < shard_v ? v : 0;
         const uint32_t tok = fdiv(vv, t.div_row);          // (bl, t) flattened
         const uint32_t col = vv - tok * t.row_v;
         const uint32_t m = fdiv(col, t.div_run);           // destination local rank
         const uint32_t j = col - m * t.run_v;
-        const uint32_t bl = fdiv(tok, p.div_T);
-        const uint32_t tt = tok - bl * p.T;
+        const uint32_t bl = fdiv(tok, div_Tr);
+        const uint32_t tt = tok - bl * Tr;
         const uint32_t hv = (bl * p.S + l * p.T + tt) * t.run_v + j;
         hrank[i] = g * p.K + m * t.rep;
         hoff[i] = hv;
@@ -90,7 +96,7 @@ __global__ void __launch_bounds__(kThreads) reshard_kernel(const __grid_constant
 #pragma unroll
     for (int i = 0; i < kUnroll; ++i) {
         const uint32_t v = v0 + i * kThreads;
-        if (v < t.shard_v) data[i] = ld_stream(kToHead ? seq + v : hp[i]);
+        if (v < shard_v) data[i] = ld_stream(kToHead ? seq + v : hp[i]);
     }
     if (!kToHead && t.rep > 1) {
         // The way back of a replicated tensor carries gradients: every copy holds the contribution of its own rank's
@@ -98,7 +104,7 @@ __global__ void __launch_bounds__(kThreads) reshard_kernel(const __grid_constant
 #pragma unroll
         for (int i = 0; i < kUnroll; ++i) {
             const uint32_t v = v0 + i * kThreads;
-            if (v >= t.shard_v) continue;
+            if (v >= shard_v) continue;
             float acc[8];
             const uint32_t w0[4] = {data[i].x, data[i].y, data[i].z, data[i].w};
 #pragma unroll
@@ -121,14 +127,14 @@ __global__ void __launch_bounds__(kThreads) reshard_kernel(const __grid_constant
 #pragma unroll
     for (int i = 0; i < kUnroll; ++i) {
         const uint32_t v = v0 + i * kThreads;
-        if (v < t.shard_v) st_stream(const_cast<uint4 *>(kToHead ? hp[i] : seq + v), data[i]);
+        if (v < shard_v) st_stream(const_cast<uint4 *>(kToHead ? hp[i] : seq + v), data[i]);
     }
     if (kToHead && t.rep > 1) {         // the other local ranks that read this KV head get the same run
         for (uint32_t c = 1; c < t.rep; ++c)
 #pragma unroll
             for (int i = 0; i < kUnroll; ++i) {
                 const uint32_t v = v0 + i * kThreads;
-                if (v < t.shard_v)
+                if (v < shard_v)
                     st_stream(const_cast<uint4 *>(reinterpret_cast<const uint4 *>(t.head[hrank[i] + c]) + hoff[i]), data[i]);
             }
     }
@@ -166,7 +172,8 @@ int fill_tensor(const basp_plan *p, const TensorArg &a, bool to_head, int r_begi
     for (int i = r_begin; i < r_begin + r_count; ++i)
         for (int j = g_begin; j < g_end; ++j) {
             const char *s = t->seq[i], *d = t->head[j];
-            if (s < d + head_bytes && d < s + shard_bytes) return BASP_ERR_ALIAS;
+            const size_t seq_bytes = shard_bytes / p->T * basp_rank_tokens(p, i % p->K);
+            if (s < d + head_bytes && d < s + seq_bytes) return BASP_ERR_ALIAS;
         }
     t->rep = (uint32_t)rep;
     t->run_v = (uint32_t)(run_bytes / 16);
@@ -188,8 +195,9 @@ int launch(const basp_plan *p, const TensorArg *args, int n, bool to_head, int r
     ReshardParams prm;
     prm.n_tensors = n;
     prm.r_begin = (uint32_t)r_begin; prm.r_count = (uint32_t)r_count;
-    prm.K = p->K; prm.T = p->T; prm.S = p->S;
+    prm.K = p->K; prm.T = p->T; prm.S = p->S; prm.Bl = p->Bl; prm.T_last = p->T_last;
     prm.div_T = make_fastdiv((uint32_t)p->T);
+    prm.div_T_last = make_fastdiv((uint32_t)p->T_last);
     uint32_t chunks = 0;
     for (int i = 0; i < n; ++i) {
         int rc = fill_tensor(p, args[i], to_head, r_begin, r_count, &prm.t[i], &chunks);

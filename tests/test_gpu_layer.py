@@ -33,6 +33,9 @@ def gpu_layer(basp, w, Xq, Xk, Xv, op, fused):
     synth.shrink(synth.WORKLOADS["sweep_b8"], 256),
     synth.shrink(synth.WORKLOADS["qwen25_7b_64k"], 128),
     synth.Workload("head_dim_96", N=4, B=2, S=512, Hq=8, Hkv=4, D=96),
+    # Table I's "Standard Ulysses (SP = N/B)" row with N = 8, B = 2: two replicas of 4 GPUs, each on its own micro-batch
+    # of 2 sequences (4 sequences in flight, B^2 S / N tokens per GPU)
+    synth.Workload("table1_sp_n_over_b", N=8, B=4, S=1024, Hq=8, Hkv=4, D=128, G=2),
 ], ids=lambda w: w.name)
 def test_layer_matches_oracle(basp, w, fused):
     Xq, Xk, Xv, op = oracle_inputs(w)

@@ -45,6 +45,18 @@ def test_plan_with_more_ranks_than_kv_heads(basp, N, B, Hq, Hkv):
         assert basp.basp_plan_get_rank(pl, r) == op.rank_info(r, Hq, Hkv)
 
 
+@pytest.mark.parametrize("N,B,G,S", [(8, 2, 0, 1022), (8, 1, 0, 1001), (4, 2, 1, 203), (8, 4, 2, 77)])
+def test_plan_for_a_length_the_group_size_does_not_divide(basp, N, B, G, S):
+    pl = basp.basp_plan_create(N, B, S, 8, 8, 64, num_groups=G)
+    op = oracle.plan_uneven(N, B, S, G)
+    assert (pl.K, pl.T, pl.T_last) == (op.K, op.T, op.T_last) and pl.T_last < pl.T
+    for r in range(N):
+        ri = basp.basp_plan_get_rank(pl, r)
+        assert (ri["token_begin"], ri["token_end"]) == op.token_range(r % op.K)
+        assert pl.rank_tokens(r) == ri["token_end"] - ri["token_begin"]
+    assert sum(pl.rank_tokens(r) for r in range(pl.K)) == S
+
+
 def test_paper_example_four_gpus_batch_two(basp):
     pl = basp.basp_plan_create(4, 2, 1024, 8, 8, 64)
     assert pl.K == 2 and [basp.basp_plan_group_ranks(pl, g) for g in range(2)] == [[0, 1], [2, 3]]
@@ -53,7 +65,7 @@ def test_paper_example_four_gpus_batch_two(basp):
 @pytest.mark.parametrize("kw,code", [
     (dict(n_ranks=8, micro_batch=3), -1),                 # N mod B != 0
     (dict(n_ranks=4, micro_batch=8), -1),                 # B > N
-    (dict(seq_len=1022), -1),                             # S mod K != 0
+    (dict(n_ranks=8, micro_batch=1, seq_len=9), -1),      # chunk = ceil(9/8) = 2 would leave the last ranks empty
     (dict(n_q_heads=30), -1),                             # Hq mod Hkv
     (dict(n_ranks=6, micro_batch=1, seq_len=1536, n_q_heads=24, n_kv_heads=4), -1),   # K = 6: neither Hkv mod K nor K mod Hkv
     (dict(num_groups=3), -1),

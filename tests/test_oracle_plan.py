@@ -41,6 +41,24 @@ def test_table1_closed_forms(N):
             assert ul.K == N and ul.Bl * ul.T == pl.Bl * pl.T == B * S // N
 
 
+@pytest.mark.parametrize("N,B", [(4, 2), (8, 2), (8, 4), (16, 4), (6, 3)])
+def test_table1_ulysses_with_sp_degree_n_over_b(N, B):
+    """Table I's middle row: standard Ulysses with sequence-parallel degree N/B.  The N GPUs form B data-parallel
+    replicas of N/B GPUs, and each replica works on a whole micro-batch of B sequences: as a plan that is B groups with B
+    sequences per group (B*B sequences in flight).  Tokens per GPU B^2 S / N, all-to-all participants N/B, as printed;
+    the same groups as BASP (which puts ONE sequence in each), B times the tokens per GPU."""
+    S = 3840
+    sp = oracle.plan(N, B * B, S, G=B)
+    basp_plan = oracle.plan(N, B, S)
+    assert sp.K == N // B == basp_plan.K                       # participants: N/B in both
+    assert sp.Bl == B and sp.Bl * sp.T == B * B * S // N       # tokens per GPU = B^2 S / N
+    assert sp.Bl * sp.T == B * basp_plan.Bl * basp_plan.T      # B times BASP's B S / N
+    assert [sp.group_ranks(g) for g in range(B)] == [basp_plan.group_ranks(g) for g in range(B)]
+    for r in range(N):
+        ri = sp.rank_info(r, Hq=N, Hkv=N)
+        assert (ri["seq_begin"], ri["seq_end"]) == (r // sp.K * B, (r // sp.K + 1) * B)   # a replica's own micro-batch
+
+
 def test_rank_info_matches_algorithm2():
     pl = oracle.plan(8, 2, 32768)
     for r in range(8):
