@@ -354,7 +354,7 @@ def run_gpu(args, w: synth.Workload):
             "clocks": clocks,
             "e2e": {"value": tokens_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
-                    "call": "basp_layer_fwd_host (fused kernel per arrived shard, copies and kernels pipelined, pinned host shards)"},
+                    "call": "basp_layer_fwd_host (fused kernel per arrived piece of query rows, copies and kernels pipelined, pinned host shards)"},
             "gpu_launches": launches,
             "roofline": {"kernel": "attn_fwd", "bound": "tensor", "achieved": attn_tflops,
                          "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",

@@ -270,11 +270,13 @@ size_t basp_layer_bwd_workspace_bytes(const basp_plan *plan);
 /* ---- the fused layer for callers whose shards are in HOST memory: copies every Q/K/V
  * shard host->device into `device_arena` (device memory, >= basp_host_arena_bytes(plan)
  * bytes), runs the fused kernel, copies every O shard device->host and waits for the stream.
- * Copies and kernels are pipelined: with the causal mask the rows of local rank l need only the
- * shards of local ranks 0..l of its group, so one launch per local rank starts as soon as that
- * shard has arrived, and its O shard is read back while later ones are still computed.  The
- * copies run on two library-owned streams (created on first use, per device; no device memory);
- * calls that overlap in time on one device share them and must be serialised by the caller.
+ * Copies and kernels are pipelined: Q travels in pieces of a few 256-row query blocks, one launch per piece
+ * starts as soon as the piece and the K and V shards it needs have arrived (with the causal mask the rows of local
+ * rank l need the shards of local ranks 0..l of its group only), and its O rows are read back while later pieces
+ * are computed; the order on the bus depends on whether the link or the GPU is the longer side (see layer.cu).
+ * Copies and kernels run on library-owned streams (created on first use, per device; no device memory) that
+ * are joined to `stream` before and after; calls that overlap in time on one device share them and must be
+ * serialised by the caller.  Needs T to be a multiple of 256 for the pipelining (else one launch per group).
  * q/k/v/o_seq_host are host arrays of n_ranks HOST pointers (pinned memory makes the copies
  * asynchronous; pageable memory works, slower). */
 int basp_layer_fwd_host(const basp_plan *plan, const void *const *q_seq_host,

@@ -35,7 +35,8 @@ namespace {
 
 template <int R>
 int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const *k, const void *const *v,
-                    void *const *o, float *const *lse, float scale, bool fused, const int range[4], cudaStream_t st) {
+                    void *const *o, float *const *lse, float scale, bool fused, const int range[4], bool cta_per_item,
+                    cudaStream_t st) {
     AttnParams<R> prm;
     const int hq = fused ? pl->Hq : pl->Hq_l, hkv = fused ? pl->Hkv : pl->Hkv_l;
     // Operands of ranks outside the launch's range are not touched: with head-sharded operands only the ranks of the
@@ -78,13 +79,17 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
         BASP_CUDA_TRY(cudaGetDevice(&dev));
         BASP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
         const long long items = (long long)range[3] * range[1] * pl->Bl * pl->Hq_l;
-        const int grid = (int)(items < sms ? items : sms);
+        // One persistent CTA per SM; a launch that shares the GPU with other launches (the pieces of the host-buffer
+        // entry) takes one CTA per item instead and leaves the balancing to the hardware's block scheduler.
+        const int grid = (int)(items < sms || (cta_per_item && items < (1 << 20)) ? items : sms);
         if (pl->D > 64) {        // 80 .. 128: the 128-wide kernel
             const int smem = (2 + kStages) * kTile * 128 * 2 + 1024;
             BASP_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_ws_kernel<128, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
             attn_fwd_ws_kernel<128, R><<<grid, kWsThreads, smem, st>>>(prm);
         } else {
-            const int smem = (2 + kStages) * kTile * 64 * 2 + 1024;
+            // every CTA holds all 512 TMEM columns: with more CTAs than SMs in flight, ask for enough shared memory that no
+            // two share an SM (the second would only sit in its TMEM allocation until the first has left)
+            const int smem = cta_per_item ? 120 * 1024 : (2 + kStages) * kTile * 64 * 2 + 1024;
             BASP_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_ws_kernel<64, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
             attn_fwd_ws_kernel<64, R><<<grid, kWsThreads, smem, st>>>(prm);
         }
@@ -101,7 +106,7 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
 // the work (NULL = everything); the host-buffer entry uses it to start on what has already arrived.
 int basp_attn_dispatch_range(const basp_plan *pl, const void *const *q, const void *const *k, const void *const *v,
                              void *const *o, float *const *lse, float scale, bool fused, const int *range,
-                             void *stream) {
+                             void *stream, bool cta_per_item) {
     if (!pl || !q || !k || !v || !o) return BASP_ERR_NULL;
     if (pl->D < 16 || pl->D > 128 || pl->D % 16 != 0) return BASP_ERR_UNSUPPORTED;
     if (fused && pl->T % kTile != 0) return BASP_ERR_UNSUPPORTED;
@@ -120,13 +125,13 @@ int basp_attn_dispatch_range(const basp_plan *pl, const void *const *q, const vo
         for (int r2 = need_lo; r2 < need_hi; ++r2)
             if (o[r] == q[r2] || o[r] == k[r2] || o[r] == v[r2]) return BASP_ERR_ALIAS;
     }
-    if (pl->N <= 8) return fill_and_launch<8>(pl, q, k, v, o, lse, scale, fused, range, (cudaStream_t)stream);
-    return fill_and_launch<BASP_MAX_RANKS>(pl, q, k, v, o, lse, scale, fused, range, (cudaStream_t)stream);
+    if (pl->N <= 8) return fill_and_launch<8>(pl, q, k, v, o, lse, scale, fused, range, cta_per_item, (cudaStream_t)stream);
+    return fill_and_launch<BASP_MAX_RANKS>(pl, q, k, v, o, lse, scale, fused, range, cta_per_item, (cudaStream_t)stream);
 }
 
 int basp_attn_dispatch(const basp_plan *pl, const void *const *q, const void *const *k, const void *const *v,
                        void *const *o, float *const *lse, float scale, bool fused, void *stream) {
-    return basp_attn_dispatch_range(pl, q, k, v, o, lse, scale, fused, nullptr, stream);
+    return basp_attn_dispatch_range(pl, q, k, v, o, lse, scale, fused, nullptr, stream, false);
 }
 
 extern "C" int basp_attn_fwd(const basp_plan *plan, const void *const *q_head, const void *const *k_head,
@@ -151,7 +156,7 @@ extern "C" int basp_attn_fwd_ranks(const basp_plan *plan, const void *const *q_h
                                    float softmax_scale, int rank_begin, int rank_count, void *stream) {
     if (!plan) return BASP_ERR_NULL;
     const int range[4] = {rank_begin, rank_count, 0, ((plan->S + kTile - 1) / kTile + 1) / 2};
-    return basp_attn_dispatch_range(plan, q_head, k_head, v_head, o_head, lse_shards, softmax_scale, false, range, stream);
+    return basp_attn_dispatch_range(plan, q_head, k_head, v_head, o_head, lse_shards, softmax_scale, false, range, stream, false);
 }
 
 extern "C" int basp_layer_fwd_fused_ranks(const basp_plan *plan, const void *const *q_seq, const void *const *k_seq,
@@ -159,5 +164,5 @@ extern "C" int basp_layer_fwd_fused_ranks(const basp_plan *plan, const void *con
                                           float softmax_scale, int rank_begin, int rank_count, void *stream) {
     if (!plan) return BASP_ERR_NULL;
     const int range[4] = {rank_begin, rank_count, 0, ((plan->S + kTile - 1) / kTile + 1) / 2};
-    return basp_attn_dispatch_range(plan, q_seq, k_seq, v_seq, o_seq, lse_shards, softmax_scale, true, range, stream);
+    return basp_attn_dispatch_range(plan, q_seq, k_seq, v_seq, o_seq, lse_shards, softmax_scale, true, range, stream, false);
 }

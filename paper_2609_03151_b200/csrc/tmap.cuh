@@ -26,8 +26,36 @@ inline EncodeTiledFn encoder() {
 
 // bf16 tensor [rows][heads][D] (D fastest) seen as 3-D (D, heads, rows); box = 64 x 1 x box_rows
 // elements with the 128-byte swizzle (each box row is one 128-byte line).
+// The encoder costs a few microseconds per map and a launch needs three maps per rank; callers that launch again and
+// again on the same buffers (a layer called every step, the pieces of the host-buffer entry) get them from a small
+// per-thread memo keyed by every argument (host memory only; a map is a pure function of its arguments).
+struct MemoEntry {
+    const void *base = nullptr;
+    uint64_t rows = 0, heads = 0, D = 0;
+    uint32_t box_rows = 0;
+    CUtensorMap map;
+};
+constexpr int kMemoSlots = 256;
+
+inline int encode_rows_heads_d_uncached(CUtensorMap *out, const void *base, uint64_t rows, uint64_t heads, uint64_t D,
+                                        uint32_t box_rows);
+
 inline int encode_rows_heads_d(CUtensorMap *out, const void *base, uint64_t rows, uint64_t heads, uint64_t D,
                                uint32_t box_rows) {
+    static thread_local MemoEntry memo[kMemoSlots];
+    const uint64_t h = ((uint64_t)(uintptr_t)base >> 8) * 0x9E3779B97F4A7C15ull + rows * 31 + heads * 7 + D + box_rows;
+    MemoEntry &e = memo[(h >> 32) % kMemoSlots];
+    if (e.base == base && e.rows == rows && e.heads == heads && e.D == D && e.box_rows == box_rows) {
+        *out = e.map;
+        return BASP_OK;
+    }
+    const int rc = encode_rows_heads_d_uncached(out, base, rows, heads, D, box_rows);
+    if (rc == BASP_OK) { e.base = base; e.rows = rows; e.heads = heads; e.D = D; e.box_rows = box_rows; e.map = *out; }
+    return rc;
+}
+
+inline int encode_rows_heads_d_uncached(CUtensorMap *out, const void *base, uint64_t rows, uint64_t heads, uint64_t D,
+                                        uint32_t box_rows) {
     EncodeTiledFn fn = encoder();
     if (!fn) {
         basp_set_cuda_error("cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)", -1, "driver entry point not found");
