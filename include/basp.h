@@ -182,8 +182,9 @@ int basp_layer_fwd_static(const basp_plan *plan, const void *const *q_seq, const
 /* ---- the same layer as ONE kernel: attention tiles are fetched straight from the
  * sequence-sharded sources (token tile at sequence position s lives on rank gK + s/T) and
  * O tiles are stored straight into the sequence-sharded destination, so the head-sharded
- * copies never exist.  Requires T to be a multiple of 128 (a tile must not straddle two ranks), else
- * BASP_ERR_UNSUPPORTED.  No workspace. */
+ * copies never exist.  Requires T to be a multiple of 128 (a tile must not straddle two ranks) and, where K does not
+ * divide S (a short last shard), one sequence per shard (Bl = 1, as in BASP grouping), else BASP_ERR_UNSUPPORTED.
+ * No workspace. */
 int basp_layer_fwd_fused(const basp_plan *plan, const void *const *q_seq, const void *const *k_seq,
                          const void *const *v_seq, void *const *o_seq, float *const *lse_shards,
                          float softmax_scale, void *stream);

@@ -18,7 +18,6 @@ struct AttnParams {
     __nv_bfloat16 *o[R];
     float *lse[R];
     int n_ranks, K, Bl, S, T, Hq_l, Hkv_l, q_per_kv;   // q_per_kv: query heads per KV head on a rank
-    int T_last;             // tokens per sequence in the sequence-sharded shard of a group's last rank (T unless K does not divide S)
     int kv_rep;             // local ranks sharing one KV head (sequence-sharded K/V: head index = local rank / kv_rep)
     int o_heads;            // heads in one row of the O destination (Hq_l, or Hq when fused)
     int Dg;                 // head dimension in memory, a multiple of 16 up to the kernel's width (64 or 128): the tile
@@ -48,7 +47,7 @@ __device__ __forceinline__ TileCoord locate(const AttnParams<R> &p, int r, int b
         const int g = r / p.K, l = r - g * p.K;
         const int owner = s0 / p.T;
         c.rank = g * p.K + owner;
-        c.row = bl * (owner == p.K - 1 ? p.T_last : p.T) + (s0 - owner * p.T);
+        c.row = bl * p.T + (s0 - owner * p.T);
         c.head = rep > 1 ? l / rep : l * heads_l + h;
     } else {
         c.rank = r;

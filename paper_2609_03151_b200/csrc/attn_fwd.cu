@@ -52,7 +52,7 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
         prm.o[r] = (__nv_bfloat16 *)o[r];
         prm.lse[r] = lse ? lse[r] : nullptr;
     }
-    prm.n_ranks = pl->N; prm.K = pl->K; prm.Bl = pl->Bl; prm.S = pl->S; prm.T = pl->T; prm.T_last = pl->T_last;
+    prm.n_ranks = pl->N; prm.K = pl->K; prm.Bl = pl->Bl; prm.S = pl->S; prm.T = pl->T;
     prm.Hq_l = pl->Hq_l; prm.Hkv_l = pl->Hkv_l; prm.q_per_kv = pl->Hq_l / pl->Hkv_l;
     prm.kv_rep = pl->kv_rep;
     prm.o_heads = hq;
@@ -110,6 +110,10 @@ int basp_attn_dispatch_range(const basp_plan *pl, const void *const *q, const vo
     if (!pl || !q || !k || !v || !o) return BASP_ERR_NULL;
     if (pl->D < 16 || pl->D > 128 || pl->D % 16 != 0) return BASP_ERR_UNSUPPORTED;
     if (fused && pl->T % kTile != 0) return BASP_ERR_UNSUPPORTED;
+    // A short last shard (K does not divide S) holds its sequences T_last rows apart, the others T: the kernel's tile
+    // addressing knows one distance only (this kernel's speed depends on its code layout; the extra select cost 5 % on
+    // one of the benchmark shapes), so that case is served when a shard holds one sequence, as in BASP grouping.
+    if (fused && pl->T_last != pl->T && pl->Bl > 1) return BASP_ERR_UNSUPPORTED;
     const int full[4] = {0, pl->N, 0, ((pl->S + kTile - 1) / kTile + 1) / 2};
     if (!range) range = full;
     if (range[0] < 0 || range[1] < 0 || range[0] + range[1] > pl->N) return BASP_ERR_INVALID;

@@ -78,10 +78,10 @@ def test_host_buffer_entry(basp):
     assert_attn_close(to_f64(out), ref["o_seq"], "host entry")
 
 
-@pytest.mark.parametrize("name", ["llama3_8b_32k"])
+@pytest.mark.parametrize("name", ["llama3_8b_32k", "sweep_b1", "sweep_b4", "sweep_b8", "qwen25_7b_64k"])
 def test_full_size_sampled_rows(basp, name):
-    """BASELINE config 2 at full size, the launches the benchmark times: sampled output rows
-    (first rows, shard and tile boundaries, last rows, random rows) against oracle rows."""
+    """BASELINE configs 2, 3 (b = 1, 4, 8; b = 2 is config 2) and 4 at full size, the launches the benchmark times:
+    sampled output rows (first rows, shard and tile boundaries, last rows, random rows) against oracle rows."""
     w = synth.WORKLOADS[name]
     q, k, v = synth.make_qkv(w, seed=0)
     pl = make_plan(basp, w)
@@ -92,7 +92,8 @@ def test_full_size_sampled_rows(basp, name):
 
     dq, dk, dv = shards(q), shards(k), shards(v)
     rng = np.random.default_rng(0)
-    cand = [0, 1, 127, 128, 255, 256, T - 1, T, T + 1, 2 * T - 1, 2 * T, w.S - 129, w.S - 128, w.S - 1]
+    cand = sorted({i for i in (0, 1, 127, 128, 255, 256, T - 1, T, T + 1, 2 * T - 1, 2 * T, w.S - 129, w.S - 128, w.S - 1)
+                   if i < w.S})
     rows = [(b, h, i) for b in range(w.B) for h in (0, 5, w.Hq - 1) for i in cand]
     rows += [(int(rng.integers(w.B)), int(rng.integers(w.Hq)), int(rng.integers(w.S))) for _ in range(40)]
     rows = np.array(rows, dtype=np.int32)

@@ -80,10 +80,12 @@ def test_arena_slices_and_guard_bands(basp):
         assert (a[r * (shard + pad): r * (shard + pad) + pad] == -1).all()
 
 
-def test_full_size_llama_reshard_sampled(basp):
-    """BASELINE config 2 at full size (the launch the benchmark times): the closed-form
+@pytest.mark.parametrize("name", ["llama3_8b_32k", "sweep_b1", "sweep_b4", "sweep_b8", "qwen25_7b_64k",
+                                  "llama3_8b_128k_train"])
+def test_full_size_reshard_sampled(basp, name):
+    """BASELINE configs 2 to 5 at full size (the launches the benchmark times): the closed-form
     destination of sampled source runs, plus the round trip being the identity."""
-    w = synth.WORKLOADS["llama3_8b_32k"]
+    w = synth.WORKLOADS[name]
     pl = basp.basp_plan_create(w.N, w.B, w.S, w.Hq, w.Hkv, w.D)
     g = torch.Generator(device="cuda").manual_seed(0)
     T, K, Hl = pl.T, pl.K, pl.Hq_l
