@@ -116,6 +116,57 @@ def plan_uneven(N: int, B: int, S: int, G: int = 0) -> Plan:
     return Plan(N=N, B=B, G=base.G, K=K, Bl=base.Bl, S=S, T=T, T_last=T_last)
 
 
+def group_sizes(N: int, B: int) -> list[int]:
+    """Ranks per group when B does not divide N.  Algorithm 1 asserts N mod B = 0 and the paper leaves the other case
+    to future work; the reading taken keeps its structure (B groups of contiguous ranks, one sequence each) and lets
+    the sizes differ by at most one: the first N mod B groups get ceil(N/B) ranks, the others floor(N/B)."""
+    if N <= 0 or B <= 0 or B > N:
+        raise ValueError(f"invalid group formation N={N} B={B}")
+    big = N % B
+    return [-(-N // B)] * big + [N // B] * (B - big)
+
+
+@dataclass(frozen=True)
+class PlanPart:
+    plan: Plan        # a uniform plan over this part's ranks and sequences
+    rank_begin: int   # first global rank of the part
+    seq_begin: int    # first sequence of the micro-batch that the part works on
+
+
+def plan_parts(N: int, B: int, S: int) -> list:
+    """The unequal groups of :func:`group_sizes` as at most two uniform plans over disjoint rank and sequence ranges:
+    the groups of ceil(N/B) ranks (ranks from 0, sequences from 0) and the groups of floor(N/B) ranks (the rest).
+    With B | N this is the one plan of Algorithm 1.  A length that a group size does not divide is cut unevenly
+    (plan_uneven)."""
+    sizes = group_sizes(N, B)
+    parts, r0, b0 = [], 0, 0
+    for K in sorted(set(sizes), reverse=True):
+        n_groups = sizes.count(K)
+        mk = plan if S % K == 0 else plan_uneven
+        parts.append(PlanPart(mk(n_groups * K, n_groups, S), r0, b0))
+        r0 += n_groups * K
+        b0 += n_groups
+    assert r0 == N and b0 == B
+    return parts
+
+
+def layer_fwd_parts(Xq: np.ndarray, Xk: np.ndarray, Xv: np.ndarray, parts: list, scale: float | None = None,
+                    causal: bool = True) -> dict:
+    """The layer over unequal groups: every part runs the layer of its own plan on its own sequences."""
+    outs = [layer_fwd(Xq[pt.seq_begin:pt.seq_begin + pt.plan.B], Xk[pt.seq_begin:pt.seq_begin + pt.plan.B],
+                      Xv[pt.seq_begin:pt.seq_begin + pt.plan.B], pt.plan, scale, causal) for pt in parts]
+    return dict(parts=outs, o_global=np.concatenate([o["o_global"] for o in outs], axis=0))
+
+
+def layer_bwd_parts(Xq, Xk, Xv, XdO, parts: list, scale: float | None = None, causal: bool = True) -> dict:
+    sl = lambda X, pt: X[pt.seq_begin:pt.seq_begin + pt.plan.B]
+    outs = [layer_bwd(sl(Xq, pt), sl(Xk, pt), sl(Xv, pt), sl(XdO, pt), pt.plan, scale, causal) for pt in parts]
+    res = dict(parts=outs)
+    for n in ("dq", "dk", "dv"):
+        res[n + "_global"] = np.concatenate([o[n + "_global"] for o in outs], axis=0)
+    return res
+
+
 # ------------------------------------------------------------------ permutations
 def _esize(a: np.ndarray) -> int:
     return int(a.dtype.itemsize)
