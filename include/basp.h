@@ -119,6 +119,25 @@ int basp_plan_get_rank(const basp_plan *plan, int rank, basp_rank_info *info);
 /* ranks_out: host array of K ints; group i is ranks i*K .. i*K+K-1 (Algorithm 1). */
 int basp_plan_group_ranks(const basp_plan *plan, int group, int *ranks_out);
 
+/* ---- group formation when B does not divide N.  Algorithm 1 asserts N mod B = 0 and the paper's limitations section
+ * leaves the other case to future work; this keeps Algorithm 1's structure (B groups of contiguous ranks, one
+ * sequence each) with sizes that differ by at most one: the first N mod B groups have ceil(N/B) ranks, the others
+ * floor(N/B).  The result is at most two PARTS, each a uniform plan over its own contiguous ranks and sequences:
+ * part 0 covers ranks [0, n_ranks_0) and sequences [0, n_seqs_0) (the larger groups), part 1 the rest.  Every other
+ * call of this header is made once per part with part.plan and with the shard arrays advanced by part.rank_begin
+ * (`shards + part.rank_begin`); the parts are independent (no exchange crosses a group), so they may run on different
+ * streams.  With N mod B = 0 there is one part, identical to basp_plan_create's plan.
+ * cfg->num_groups must be 0 or equal to micro_batch (BASP grouping).  Errors: as basp_plan_create for each part
+ * (e.g. BASP_ERR_INVALID when a group size divides neither head count); B > N is BASP_ERR_INVALID.  On success the
+ * caller owns parts[i].plan for i < *n_parts (basp_plan_destroy). */
+typedef struct basp_plan_part {
+    basp_plan *plan;
+    int rank_begin, n_ranks;   /* global ranks [rank_begin, rank_begin + n_ranks)            */
+    int seq_begin, n_seqs;     /* sequences of the micro-batch [seq_begin, seq_begin + n_seqs) */
+    int group_size;            /* ranks per group in this part                               */
+} basp_plan_part;
+int basp_plan_create_parts(const basp_config *cfg, basp_plan_part parts[2], int *n_parts);
+
 /* ---- reshards: the two all-to-alls of the Ulysses layer confined to each group
  * (Section II-C, Section IV-C), as out-of-place permutations inside device memory.
  *   s2h: head[gK+m][bl][s][h'][d] = seq[gK + s/T][bl][s mod T][m*H/K + h'][d]

@@ -31,7 +31,7 @@ EXPORTS = [
     "basp_layer_bwd", "basp_layer_bwd_workspace_bytes", "basp_get_status", "basp_clear_status",
     "basp_strerror", "basp_last_cuda_error", "basp_launch_count", "basp_selftest_wait_timeout", "basp_qkv_proj", "basp_out_proj",
     "basp_reshard_qkv_s2h_ranks", "basp_reshard_h2s_ranks", "basp_attn_fwd_ranks", "basp_layer_fwd_fused_ranks",
-    "basp_qkv_proj_rope", "basp_layer_bwd_seq", "basp_layer_bwd_seq_workspace_bytes",
+    "basp_qkv_proj_rope", "basp_layer_bwd_seq", "basp_layer_bwd_seq_workspace_bytes", "basp_plan_create_parts",
 ]
 
 
@@ -155,6 +155,40 @@ def basp_plan_create(n_ranks, micro_batch, seq_len, n_q_heads, n_kv_heads, head_
     out = c_void_p()
     _check(lib.basp_plan_create(byref(cfg), byref(out)), "basp_plan_create")
     return Plan(out.value, cfg)
+
+
+class basp_plan_part(Structure):
+    _fields_ = [("plan", c_void_p)] + [(n, c_int) for n in ("rank_begin", "n_ranks", "seq_begin", "n_seqs", "group_size")]
+
+
+lib.basp_plan_create_parts.argtypes = [POINTER(basp_config), POINTER(basp_plan_part), POINTER(c_int)]
+
+
+class PlanPart:
+    """One uniform part of an unequal group formation: `plan` serves global ranks [rank_begin, rank_begin + n_ranks)
+    and sequences [seq_begin, seq_begin + n_seqs); `shards(x)` cuts a per-rank list down to the part's ranks."""
+
+    def __init__(self, plan: Plan, rank_begin: int, n_ranks: int, seq_begin: int, n_seqs: int, group_size: int):
+        self.plan, self.rank_begin, self.n_ranks = plan, rank_begin, n_ranks
+        self.seq_begin, self.n_seqs, self.group_size = seq_begin, n_seqs, group_size
+
+    def shards(self, per_rank):
+        return list(per_rank[self.rank_begin:self.rank_begin + self.n_ranks])
+
+
+def basp_plan_create_parts(n_ranks, micro_batch, seq_len, n_q_heads, n_kv_heads, head_dim, causal=True, dtype=0):
+    """Group formation for any micro_batch <= n_ranks (groups of ceil and floor(N/B) ranks): a list of one or two
+    PlanPart.  Every call of the library is then made per part with part.plan and part.shards(...)."""
+    cfg = basp_config(n_ranks, micro_batch, 0, seq_len, n_q_heads, n_kv_heads, head_dim, dtype, int(causal))
+    arr = (basp_plan_part * 2)()
+    n = c_int(0)
+    _check(lib.basp_plan_create_parts(byref(cfg), arr, byref(n)), "basp_plan_create_parts")
+    out = []
+    for i in range(n.value):
+        c = basp_config(arr[i].n_ranks, arr[i].n_seqs, 0, seq_len, n_q_heads, n_kv_heads, head_dim, dtype, int(causal))
+        out.append(PlanPart(Plan(arr[i].plan, c), arr[i].rank_begin, arr[i].n_ranks, arr[i].seq_begin, arr[i].n_seqs,
+                            arr[i].group_size))
+    return out
 
 
 def basp_plan_get_rank(plan: Plan, rank: int) -> dict:

@@ -39,6 +39,39 @@ extern "C" int basp_plan_create(const basp_config *cfg, basp_plan **out) {
     return BASP_OK;
 }
 
+// Unequal groups (B does not divide N): the first N mod B groups take ceil(N/B) ranks, the others floor(N/B); each
+// size class is a uniform plan of its own over a contiguous range of ranks and sequences.
+extern "C" int basp_plan_create_parts(const basp_config *cfg, basp_plan_part parts[2], int *n_parts) {
+    if (!cfg || !parts || !n_parts) return BASP_ERR_NULL;
+    *n_parts = 0;
+    parts[0].plan = parts[1].plan = nullptr;
+    const int N = cfg->n_ranks, B = cfg->micro_batch;
+    if (N <= 0 || B <= 0 || B > N) return BASP_ERR_INVALID;
+    if (cfg->num_groups != 0 && cfg->num_groups != B) return BASP_ERR_INVALID;
+    const int big = N % B, k_hi = (N + B - 1) / B, k_lo = N / B;
+    const int groups[2] = {big == 0 ? B : big, big == 0 ? 0 : B - big};
+    const int sizes[2] = {big == 0 ? k_lo : k_hi, k_lo};
+    int r0 = 0, b0 = 0;
+    for (int i = 0; i < 2 && groups[i] > 0; ++i) {
+        basp_config c = *cfg;
+        c.n_ranks = groups[i] * sizes[i];
+        c.micro_batch = groups[i];
+        c.num_groups = 0;
+        const int rc = basp_plan_create(&c, &parts[i].plan);
+        if (rc != BASP_OK) {
+            if (i == 1) { basp_plan_destroy(parts[0].plan); parts[0].plan = nullptr; }
+            *n_parts = 0;
+            return rc;
+        }
+        parts[i].rank_begin = r0; parts[i].n_ranks = c.n_ranks;
+        parts[i].seq_begin = b0; parts[i].n_seqs = groups[i];
+        parts[i].group_size = sizes[i];
+        r0 += c.n_ranks; b0 += groups[i];
+        *n_parts = i + 1;
+    }
+    return BASP_OK;
+}
+
 extern "C" int basp_plan_destroy(basp_plan *plan) {
     if (!plan) return BASP_ERR_NULL;
     delete plan;

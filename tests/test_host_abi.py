@@ -57,6 +57,31 @@ def test_plan_for_a_length_the_group_size_does_not_divide(basp, N, B, G, S):
     assert sum(pl.rank_tokens(r) for r in range(pl.K)) == S
 
 
+@pytest.mark.parametrize("N,B", [(8, 3), (8, 5), (7, 2), (7, 3), (6, 4), (8, 2), (5, 5)])
+def test_unequal_group_formation_matches_oracle(basp, N, B):
+    S, Hq = 840, 840                                   # divisible by every group size that occurs
+    parts = basp.basp_plan_create_parts(N, B, S, Hq, Hq, 16)
+    want = oracle.plan_parts(N, B, S)
+    assert len(parts) == len(want)
+    for got, ref in zip(parts, want):
+        assert (got.rank_begin, got.n_ranks, got.seq_begin, got.n_seqs) == (ref.rank_begin, ref.plan.N, ref.seq_begin, ref.plan.B)
+        assert (got.plan.K, got.plan.G, got.plan.Bl, got.plan.T) == (ref.plan.K, ref.plan.G, 1, ref.plan.T)
+        assert got.group_size == ref.plan.K
+    assert [p.group_size for p in parts for _ in range(p.n_seqs)] == oracle.group_sizes(N, B)
+    if N % B == 0:
+        whole = basp.basp_plan_create(N, B, S, Hq, Hq, 16)
+        assert len(parts) == 1 and (parts[0].plan.K, parts[0].plan.T) == (whole.K, whole.T)
+
+
+def test_unequal_group_formation_errors(basp):
+    with pytest.raises(basp.BaspError) as e:
+        basp.basp_plan_create_parts(4, 5, 1024, 8, 8, 64)          # more sequences than ranks
+    assert e.value.code == basp.BASP_ERR_INVALID
+    with pytest.raises(basp.BaspError) as e:
+        basp.basp_plan_create_parts(8, 3, 1536, 8, 8, 64)          # groups of 3 ranks cannot split 8 heads
+    assert e.value.code == basp.BASP_ERR_INVALID
+
+
 def test_paper_example_four_gpus_batch_two(basp):
     pl = basp.basp_plan_create(4, 2, 1024, 8, 8, 64)
     assert pl.K == 2 and [basp.basp_plan_group_ranks(pl, g) for g in range(2)] == [[0, 1], [2, 3]]
