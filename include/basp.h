@@ -97,8 +97,10 @@ typedef struct basp_rank_info {
 /* ---- plan: Algorithm 1 (K = N/B, contiguous rank blocks, N mod B = 0 asserted) and
  * Algorithm 2 (group = r / K, local = r mod K, chunk = S / K), generalised to G groups
  * as in the workload-equivalence paragraph of Section IV-C.
- * Errors: BASP_ERR_NULL; BASP_ERR_INVALID for N mod G != 0, B mod G != 0, B > N in BASP
- * mode (the paper's data-parallel fallback is not provided), an empty last rank (below), Hq mod Hkv != 0,
+ * With num_groups = 0 and B > N the plan is the paper's data-parallel fallback: N groups of one rank (K = 1), B/N whole
+ * sequences per rank, both exchanges identities.
+ * Errors: BASP_ERR_NULL; BASP_ERR_INVALID for N mod G != 0, B mod G != 0 (so B > N needs N | B), an empty last rank
+ * (below), Hq mod Hkv != 0,
  * Hq mod K != 0, or Hkv and K with neither Hkv mod K = 0 nor K mod Hkv = 0; BASP_ERR_UNSUPPORTED for
  * dtype != bf16, N > BASP_MAX_RANKS or a head slice whose row ((H/K)*D*2 bytes) is not a multiple of 16 bytes.
  * A group with MORE ranks than KV heads (K mod Hkv = 0, K > Hkv; the paper does not treat grouped-query attention)
@@ -128,7 +130,7 @@ int basp_plan_group_ranks(const basp_plan *plan, int group, int *ranks_out);
  * (`shards + part.rank_begin`); the parts are independent (no exchange crosses a group), so they may run on different
  * streams.  With N mod B = 0 there is one part, identical to basp_plan_create's plan.
  * cfg->num_groups must be 0 or equal to micro_batch (BASP grouping).  Errors: as basp_plan_create for each part
- * (e.g. BASP_ERR_INVALID when a group size divides neither head count); B > N is BASP_ERR_INVALID.  On success the
+ * (e.g. BASP_ERR_INVALID when a group size divides neither head count); B > N gives the one data-parallel plan.  On success the
  * caller owns parts[i].plan for i < *n_parts (basp_plan_destroy). */
 typedef struct basp_plan_part {
     basp_plan *plan;

@@ -44,9 +44,10 @@ int oracle_num_threads(void) {
  * Returns 0 when valid, -1 otherwise.  out = {K, G, Bl, T}. */
 int oracle_plan(int N, int B, int G, int S, int out[4]) {
     if (N <= 0 || B <= 0 || S <= 0) return -1;
-    if (G == 0) G = B;              /* BASP: one group per sequence          */
+    /* BASP: one group per sequence.  More sequences than ranks: the paper's fallback to plain data parallelism,
+     * i.e. every rank a group of its own (K = 1) that holds B/N whole sequences. */
+    if (G == 0) G = B > N ? N : B;
     if (G <= 0) return -1;
-    if (B > N && G == B) return -1; /* B > N is the data-parallel fallback   */
     if (N % G != 0) return -1;      /* "assert N mod B = 0"                  */
     if (B % G != 0) return -1;
     int K = N / G;

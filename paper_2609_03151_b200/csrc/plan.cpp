@@ -12,8 +12,9 @@ extern "C" int basp_plan_create(const basp_config *cfg, basp_plan **out) {
     const int Hq = cfg->n_q_heads, Hkv = cfg->n_kv_heads, D = cfg->head_dim;
     if (N <= 0 || B <= 0 || S <= 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || cfg->num_groups < 0)
         return BASP_ERR_INVALID;
-    const int G = cfg->num_groups == 0 ? B : cfg->num_groups;   // Algorithm 1: num_groups = B
-    if (G == B && B > N) return BASP_ERR_INVALID;               // data-parallel fallback: not a plan
+    // Algorithm 1: num_groups = B.  With more sequences than ranks the method falls back to plain data parallelism
+    // (Section IV-B): every rank is a group of its own (K = 1) holding B/N whole sequences; the exchanges are identities.
+    const int G = cfg->num_groups == 0 ? (B > N ? N : B) : cfg->num_groups;
     if (N % G != 0 || B % G != 0) return BASP_ERR_INVALID;      // Algorithm 1: assert N mod B = 0
     const int K = N / G;                                         // Algorithm 1: K = N / B
     // Algorithm 2: chunk = L / K.  Where K does not divide L (the paper is silent) the chunk is rounded up and the
@@ -46,8 +47,17 @@ extern "C" int basp_plan_create_parts(const basp_config *cfg, basp_plan_part par
     *n_parts = 0;
     parts[0].plan = parts[1].plan = nullptr;
     const int N = cfg->n_ranks, B = cfg->micro_batch;
-    if (N <= 0 || B <= 0 || B > N) return BASP_ERR_INVALID;
+    if (N <= 0 || B <= 0) return BASP_ERR_INVALID;
     if (cfg->num_groups != 0 && cfg->num_groups != B) return BASP_ERR_INVALID;
+    if (B > N) {                              // the data-parallel fallback is one uniform plan
+        basp_config c = *cfg;
+        c.num_groups = 0;
+        const int rc = basp_plan_create(&c, &parts[0].plan);
+        if (rc != BASP_OK) return rc;
+        parts[0].rank_begin = 0; parts[0].n_ranks = N; parts[0].seq_begin = 0; parts[0].n_seqs = B; parts[0].group_size = 1;
+        *n_parts = 1;
+        return BASP_OK;
+    }
     const int big = N % B, k_hi = (N + B - 1) / B, k_lo = N / B;
     const int groups[2] = {big == 0 ? B : big, big == 0 ? 0 : B - big};
     const int sizes[2] = {big == 0 ? k_lo : k_hi, k_lo};

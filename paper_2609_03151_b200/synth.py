@@ -27,7 +27,7 @@ class Workload:
 
     @property
     def K(self) -> int:
-        return self.N // (self.G or self.B)
+        return self.N // (self.G or min(self.B, self.N))     # more sequences than ranks: one rank per group
 
     @property
     def tokens(self) -> int:

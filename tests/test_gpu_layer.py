@@ -36,6 +36,8 @@ def gpu_layer(basp, w, Xq, Xk, Xv, op, fused):
     # Table I's "Standard Ulysses (SP = N/B)" row with N = 8, B = 2: two replicas of 4 GPUs, each on its own micro-batch
     # of 2 sequences (4 sequences in flight, B^2 S / N tokens per GPU)
     synth.Workload("table1_sp_n_over_b", N=8, B=4, S=1024, Hq=8, Hkv=4, D=128, G=2),
+    # more sequences than ranks: the data-parallel fallback (one rank per group, two whole sequences each)
+    synth.Workload("data_parallel_fallback", N=4, B=8, S=512, Hq=4, Hkv=2, D=64),
 ], ids=lambda w: w.name)
 def test_layer_matches_oracle(basp, w, fused):
     Xq, Xk, Xv, op = oracle_inputs(w)

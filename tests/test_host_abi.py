@@ -75,11 +75,21 @@ def test_unequal_group_formation_matches_oracle(basp, N, B):
 
 def test_unequal_group_formation_errors(basp):
     with pytest.raises(basp.BaspError) as e:
-        basp.basp_plan_create_parts(4, 5, 1024, 8, 8, 64)          # more sequences than ranks
+        basp.basp_plan_create_parts(4, 5, 1024, 8, 8, 64)          # more sequences than ranks, and 4 does not divide 5
     assert e.value.code == basp.BASP_ERR_INVALID
+    (dp,) = basp.basp_plan_create_parts(4, 8, 1024, 8, 8, 64)      # the data-parallel fallback is one part
+    assert (dp.plan.K, dp.plan.Bl, dp.n_ranks, dp.n_seqs) == (1, 2, 4, 8)
     with pytest.raises(basp.BaspError) as e:
         basp.basp_plan_create_parts(8, 3, 1536, 8, 8, 64)          # groups of 3 ranks cannot split 8 heads
     assert e.value.code == basp.BASP_ERR_INVALID
+
+
+def test_data_parallel_fallback_plan(basp):
+    pl = basp.basp_plan_create(4, 8, 1024, 8, 8, 64)                 # B > N: one rank per group, two whole sequences each
+    op = oracle.plan(4, 8, 1024)
+    assert (pl.K, pl.G, pl.Bl, pl.T) == (op.K, op.G, op.Bl, op.T) == (1, 4, 2, 1024)
+    for r in range(4):
+        assert basp.basp_plan_get_rank(pl, r) == op.rank_info(r, 8, 8)
 
 
 def test_paper_example_four_gpus_batch_two(basp):
@@ -89,7 +99,7 @@ def test_paper_example_four_gpus_batch_two(basp):
 
 @pytest.mark.parametrize("kw,code", [
     (dict(n_ranks=8, micro_batch=3), -1),                 # N mod B != 0
-    (dict(n_ranks=4, micro_batch=8), -1),                 # B > N
+    (dict(n_ranks=4, micro_batch=6), -1),                 # B > N and N does not divide B
     (dict(n_ranks=8, micro_batch=1, seq_len=9), -1),      # chunk = ceil(9/8) = 2 would leave the last ranks empty
     (dict(n_q_heads=30), -1),                             # Hq mod Hkv
     (dict(n_ranks=6, micro_batch=1, seq_len=1536, n_q_heads=24, n_kv_heads=4), -1),   # K = 6: neither Hkv mod K nor K mod Hkv

@@ -1,6 +1,7 @@
 """Pins of the oracle's plan against what the paper fixes (Algorithms 1 and 2, Table I)."""
 import os
 
+import numpy as np
 import pytest
 
 import oracle
@@ -70,9 +71,24 @@ def test_rank_info_matches_algorithm2():
         assert (ri["kv_head_begin"], ri["kv_head_end"]) == ((r % 4) * 2, (r % 4 + 1) * 2)
 
 
+def test_more_sequences_than_ranks_falls_back_to_data_parallelism():
+    """Section IV-B: with B > N there is nothing to shard; every rank takes whole sequences (K = 1, B/N of them)."""
+    pl = oracle.plan(4, 8, 1024)
+    assert (pl.K, pl.G, pl.Bl, pl.T) == (1, 4, 2, 1024)
+    for r in range(4):
+        ri = pl.rank_info(r, Hq=8, Hkv=8)
+        assert (ri["group"], ri["local_rank"]) == (r, 0)
+        assert (ri["seq_begin"], ri["seq_end"]) == (2 * r, 2 * r + 2)
+        assert (ri["token_begin"], ri["token_end"]) == (0, 1024) and (ri["q_head_begin"], ri["q_head_end"]) == (0, 8)
+    X = np.arange(8 * 1024 * 8 * 2, dtype=np.int32).reshape(8, 1024, 8, 2)
+    seq = oracle.partition(X, pl)
+    assert np.array_equal(seq.reshape(X.shape), X)                 # rank r holds sequences 2r, 2r+1 whole
+    assert np.array_equal(oracle.s2h(seq, pl), seq)                # the exchange of a one-rank group is the identity
+
+
 @pytest.mark.parametrize("N,B,S,G", [
     (8, 3, 1024, 0),     # N mod B != 0 (Algorithm 1's assertion)
-    (4, 8, 1024, 0),     # B > N: data-parallel fallback, not a sequence-parallel plan
+    (4, 6, 1024, 0),     # B > N and N does not divide B: no data-parallel split either
     (8, 2, 1022, 0),     # S not divisible by K
     (8, 4, 1024, 3),     # G does not divide N / B
     (0, 1, 1024, 0),
