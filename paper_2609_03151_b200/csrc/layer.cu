@@ -157,6 +157,7 @@ struct HostPipe {
     }
 };
 constexpr int kHostPieceWaves = 2;
+constexpr int kHostUpperEighths = 5;   // share of a group's pieces (from the end of the sequence) sent right behind its K and V
 // Sustained attention rate over host-link rate of the machine this was tuned on (about 1.3 PFLOP/s over 50 GB/s).
 constexpr double kHostBalanceFlopPerByte = 26e3;
 std::mutex g_pipe_mu;
@@ -189,9 +190,10 @@ int get_pipe(HostPipe **out) {
 // long-sequence shapes, so the order on the bus is chosen to start the GPU early and never let it run dry.  A group's
 // K and V shards go first (a quarter of the bytes under GQA; every query row needs a prefix of them), then its Q rows
 // in PIECES of a few 256-row query blocks from the END of the sequence down: under the causal mask a piece's arithmetic
-// grows with its position, so the first pieces carry the most work per byte.  After the UPPER half of a group's pieces
-// (three quarters of its arithmetic) the next group's K and V and upper half follow, the backlog on the GPU covering
-// the K/V transfer; the cheap lower halves of all groups come last, which keeps the tail behind the last byte short.
+// grows with its position, so the first pieces carry the most work per byte.  After the UPPER 5/8 of a group's pieces
+// (most of its arithmetic) the next group's K and V and upper pieces follow, the backlog on the GPU covering the K/V
+// transfer; the cheap lower pieces of a group travel between the next group's upper pieces (their O rows leave early
+// instead of queueing behind the last byte), the last group's lower pieces come last: a short tail.
 // One launch per piece (all ranks and heads of the group, the piece's query blocks, one CTA per work item so that
 // consecutive launches fill each other's last wave) starts as soon as the piece is there, and its O rows are read back
 // while later pieces run.
@@ -268,10 +270,18 @@ extern "C" int basp_layer_fwd_host(const basp_plan *p, const void *const *q_seq_
                 continue;
             }
             // The bus is the longer side (or they balance): every group's pieces from the end of its sequences down; the
-            // upper half of group 0's pieces, of group 1's, ... each behind its group's K and V, the lower halves of all
-            // groups at the end.
-            const size_t upper = p->causal ? (mine.size() + 1) / 2 : mine.size();
-            pieces.insert(pieces.end(), mine.begin(), mine.begin() + upper);
+            // upper 5/8 of a group's pieces right behind its K and V, its lower pieces woven into the next group's upper
+            // ones, the last group's lower pieces at the end.
+            const size_t upper = p->causal ? (mine.size() * kHostUpperEighths + 7) / 8 : mine.size();
+            // the previous group's cheap lower pieces travel between this group's upper pieces, one for one: their O rows
+            // leave early instead of queueing on the way out behind the last byte
+            size_t li = 0;
+            for (size_t i = 0; i < upper; ++i) {
+                pieces.push_back(mine[i]);
+                if (li < lower.size()) pieces.push_back(lower[li++]);
+            }
+            pieces.insert(pieces.end(), lower.begin() + li, lower.end());
+            lower.clear();
             lower.insert(lower.end(), mine.begin() + upper, mine.end());
         }
         pieces.insert(pieces.end(), lower.begin(), lower.end());
