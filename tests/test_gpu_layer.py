@@ -66,11 +66,16 @@ def test_tiny_basp_equals_ulysses_equals_unpartitioned(basp):
         assert np.array_equal(val, first), key
 
 
-def test_host_buffer_entry(basp):
-    w = synth.shrink(synth.WORKLOADS["llama3_8b_32k"], 128)
+@pytest.mark.parametrize("w,causal", [
+    (synth.shrink(synth.WORKLOADS["llama3_8b_32k"], 128), True),                          # T = 128: one launch per group
+    (synth.Workload("pieces_two_groups", N=8, B=2, S=4096, Hq=8, Hkv=4, D=128), True),    # T = 1024: several pieces per shard
+    (synth.Workload("pieces_d64_two_seqs", N=4, B=4, S=2048, Hq=4, Hkv=2, D=64, G=2), True),   # D = 64, two sequences per group
+    (synth.Workload("pieces_unmasked", N=4, B=2, S=1024, Hq=4, Hkv=4, D=64), False),      # every piece needs all of K and V
+], ids=lambda x: getattr(x, "name", str(x)))
+def test_host_buffer_entry(basp, w, causal):
     Xq, Xk, Xv, op = oracle_inputs(w, seed=2)
-    ref = oracle.layer_fwd(Xq, Xk, Xv, op)
-    pl = make_plan(basp, w)
+    ref = oracle.layer_fwd(Xq, Xk, Xv, op, causal=causal)
+    pl = make_plan(basp, w, causal=causal)
     host = [[synth.from_bits(a[r]).pin_memory() for r in range(w.N)] for a in (ref["q_seq"], ref["k_seq"], ref["v_seq"])]
     out = [torch.zeros_like(t).pin_memory() for t in host[0]]
     arena = torch.empty(basp.basp_host_arena_bytes(pl), dtype=torch.uint8, device="cuda")
@@ -78,6 +83,32 @@ def test_host_buffer_entry(basp):
     basp.basp_layer_fwd_host(pl, host[0], host[1], host[2], out, arena)
     basp.basp_get_status()
     assert_attn_close(to_f64(out), ref["o_seq"], "host entry")
+
+
+@pytest.mark.parametrize("name", ["llama3_8b_32k", "sweep_b1"])
+def test_host_buffer_entry_full_size_sampled_rows(basp, name):
+    """The host-buffer entry at full size, in both orders of its pipeline (config 2: the link is the longer side; config 3
+    at b = 1: the GPU is), on sampled output rows."""
+    w = synth.WORKLOADS[name]
+    q, k, v = synth.make_qkv(w, seed=0)
+    pl = make_plan(basp, w)
+    T, K = pl.T, pl.K
+    cut = lambda x: [x[r // K: r // K + 1, (r % K) * T:(r % K + 1) * T].contiguous().pin_memory() for r in range(w.N)]
+    hq, hk, hv = cut(q), cut(k), cut(v)
+    ho = [torch.full_like(t, float("nan")).pin_memory() for t in hq]
+    arena = torch.empty(basp.basp_host_arena_bytes(pl), dtype=torch.uint8, device="cuda")
+    basp.basp_clear_status()
+    basp.basp_layer_fwd_host(pl, hq, hk, hv, ho, arena)
+    basp.basp_get_status()
+    assert not any(torch.isnan(t.float()).any() for t in ho)                 # every row of every shard came back
+    rng = np.random.default_rng(1)
+    cand = [0, 255, 256, 2047, 2048, T - 1, T, 2 * T - 1, 2 * T, w.S - 2049, w.S - 2048, w.S - 1]
+    rows = [(b, h, i) for b in range(w.B) for h in (0, w.Hq - 1) for i in cand]
+    rows += [(int(rng.integers(w.B)), int(rng.integers(w.Hq)), int(rng.integers(w.S))) for _ in range(40)]
+    rows = np.array(rows, dtype=np.int32)
+    ref, _ = oracle.attn_fwd_rows(synth.bits(q), synth.bits(k), synth.bits(v), rows)
+    got = np.stack([ho[b * K + i // T][0, i % T, h].float().numpy().astype(np.float64) for b, h, i in rows])
+    assert_attn_close(got, ref, f"{name} host entry")
 
 
 @pytest.mark.parametrize("name", ["llama3_8b_32k", "sweep_b1", "sweep_b4", "sweep_b8", "qwen25_7b_64k"])
