@@ -308,6 +308,24 @@ def run_gpu(args, w: synth.Workload):
     torch.cuda.synchronize()
     ms_fused = f0.elapsed_time(f1) / args.steps
     basp.basp_get_status()
+
+    # the same three launches replayed from a CUDA graph (the calls are capturable: asynchronous, no allocation, no
+    # synchronisation): what the step costs without the host's launch path, which is what config 1 is bound by
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        step()
+    graph.replay()
+    torch.cuda.synchronize()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record()
+    for _ in range(args.steps):
+        graph.replay()
+    g1.record()
+    torch.cuda.synchronize()
+    ms_graph = g0.elapsed_time(g1) / args.steps
+    basp.basp_get_status()
+    del graph
     clocks = sampler.stop() if sampler else None
 
     # end to end through the C ABI with HOST buffers: H2D of Q, K, V and D2H of O inside the timed region
@@ -372,6 +390,8 @@ def run_gpu(args, w: synth.Workload):
             },
             "fused": {"ms_per_step": ms_fused_max, "value": tokens_all / (ms_fused_max * 1e-3), "unit": UNIT,
                       "tflops": flops / (ms_fused * 1e-3) / 1e12, "launches_per_step": 1},
+            "graph_replay": {"ms_per_step": ms_graph, "value": w.tokens / (ms_graph * 1e-3), "unit": UNIT,
+                             "what": "the step's three launches captured once into a CUDA graph and replayed"},
             "cpu_baseline": cpu,
         }
         print(json.dumps(line), flush=True)
