@@ -14,7 +14,8 @@ pytestmark = pytest.mark.gpu
     synth.shrink(synth.WORKLOADS["llama3_8b_32k"], 128),
     synth.Workload("tiny_like_d64", N=4, B=2, S=512, Hq=8, Hkv=8, D=64),
 ], ids=lambda w: w.name)
-def test_autograd_matches_oracle(basp, w):
+@pytest.mark.parametrize("fused", [False, True])
+def test_autograd_matches_oracle(basp, w, fused):
     from paper_2609_03151_b200.autograd import basp_attention
     q, k, v, do_ = synth.make_qkv(w, seed=5, with_dO=True)
     Xq, Xk, Xv, Xdo = (synth.bits(t) for t in (q, k, v, do_))
@@ -25,7 +26,7 @@ def test_autograd_matches_oracle(basp, w):
     qs, ks, vs = ([t.requires_grad_() for t in to_dev(oracle.partition(X, op))] for X in (Xq, Xk, Xv))
     dos = to_dev(oracle.partition(Xdo, op))
     basp.basp_clear_status()
-    o = basp_attention(pl, qs, ks, vs)
+    o = basp_attention(pl, qs, ks, vs, fused=fused)
     torch.autograd.backward(o, dos)
     basp.basp_get_status()
     assert_attn_close(to_f64([t.detach() for t in o]), ref_f["o_seq"], w.name)
