@@ -112,17 +112,21 @@ __device__ long long g_bwd_phase[32];
         }                                                                       \
     } while (0)
 
-template <int R>
+// D = 128 or 64: the kernel's width (columns of the Q, K, V, dO tiles and of the dQ, dK, dV accumulators).  A tile is D/64
+// slabs of [128 rows][64 columns] (one 128-byte swizzled line per row and slab).
+template <int D, int R>
 __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_constant__ BwdParams<R> p) {
-    constexpr int D = 128;
-    constexpr int kTileBytes = kT * D * 2;             // 32 KiB
+    static_assert(D == 64 || D == 128, "kernel widths");
+    constexpr int kSlabs = D / 64;
+    constexpr int kTileBytes = kT * D * 2;             // 32 KiB (16 KiB at D = 64)
+    constexpr int kDqChunks = D / 32;                  // 32-column fp32 chunks of a dQ tile
     // dynamic shared memory only, so that the tile area starts at the (1024-byte aligned) window base
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t *sK = smem, *sV = smem + kTileBytes;
     uint8_t *sQ = smem + 2 * kTileBytes;               // 2 stages
     uint8_t *sdO = smem + 4 * kTileBytes;              // 2 stages
-    uint8_t *sdS = smem + 6 * kTileBytes;              // dS^T [key rows][query cols], two 64-column slabs
-    float *s_lse = reinterpret_cast<float *>(smem + 7 * kTileBytes);   // [2][128], already times log2(e)
+    uint8_t *sdS = smem + 6 * kTileBytes;              // dS^T [key rows][query cols], two 64-column slabs (32 KiB)
+    float *s_lse = reinterpret_cast<float *>(sdS + 2 * 16384);         // [2][128], already times log2(e)
     float *s_delta = s_lse + 2 * kT;                                   // [2][128]
     BwdBars *bars = reinterpret_cast<BwdBars *>(s_delta + 2 * kT);
 
@@ -249,13 +253,14 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             BWD_WAIT(&bars->dkdv_full, item_n & 1, 13, item.n);
             tc_fence_after();
             {
-                // quarters 0,1 write the two 64-column halves of dK, quarters 2,3 those of dV
+                // quarters 0,1 write the two halves (D/2 columns each) of dK, quarters 2,3 those of dV
+                constexpr int kHalf = D / 2;
                 __nv_bfloat16 *base = (g < 2 ? p.dk[item.r] : p.dv[item.r]) +
                                       (((size_t)item.bl * p.S + (size_t)item.n * kT + row) * p.Hkv_l + item.hkv) * p.Dg +
-                                      64 * (g & 1);
-                const uint32_t col0 = (g < 2 ? kColDK : kColDV) + 64 * (g & 1);
+                                      kHalf * (g & 1);
+                const uint32_t col0 = (g < 2 ? kColDK : kColDV) + kHalf * (g & 1);
 #pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
+                for (int cc = 0; cc < kHalf / 32; ++cc) {
                     uint32_t rr[32];
                     tmem_ld_x32(tmem + col0 + cc * 32 + lane_addr, rr);
                     tmem_wait_ld();
@@ -266,7 +271,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                         o4.y = pack_bf16x2(__uint_as_float(rr[8 * i + 2]), __uint_as_float(rr[8 * i + 3]));
                         o4.z = pack_bf16x2(__uint_as_float(rr[8 * i + 4]), __uint_as_float(rr[8 * i + 5]));
                         o4.w = pack_bf16x2(__uint_as_float(rr[8 * i + 6]), __uint_as_float(rr[8 * i + 7]));
-                        if (64 * (g & 1) + cc * 32 + i * 8 < p.Dg && item.n * kT + row < p.S)
+                        if (kHalf * (g & 1) + cc * 32 + i * 8 < p.Dg && item.n * kT + row < p.S)
                             *reinterpret_cast<uint4 *>(base + cc * 32 + i * 8) = o4;
                     }
                 }
@@ -277,10 +282,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         }
     } else if (warp < kBwdTmaWarp) {
         // ======================================================================= dQ drain warps
-        // dQ_m (lane = query row, 128 fp32 columns) leaves TMEM through the Q / dO stage of its step, which is
-        // 64 KiB of free shared memory once the products that read it are done: chunk c ([128 rows][32 floats],
-        // 128-byte swizzle) goes to the dO half (c = 2, 3; product (3) is complete when dQ is) or the Q half
-        // (c = 0, 1; after product (4)).  Each warp adds its 32 rows of a chunk with one TMA reduce-add.
+        // dQ_m (lane = query row, D fp32 columns) leaves TMEM through the Q / dO stage of its step, which is free
+        // shared memory of exactly its size once the products that read it are done: chunk c ([128 rows][32 floats],
+        // 128-byte swizzle) goes to the dO half (the upper half of the chunks; product (3) is complete when dQ is) or
+        // the Q half (the lower half; after product (4)).  Each warp adds its 32 rows of a chunk with one TMA reduce-add.
         reg_inc<104>();
         const int wq = warp & 3;
         const int row = tid & 127;
@@ -296,9 +301,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     BWD_WAIT(&bars->dq_full, it_g & 1, 12, m);
                     tc_fence_after();
                     BPH_T(v1);
-                    uint32_t lo[64];
+                    constexpr int kHalfCh = kDqChunks / 2;            // chunks per half: 2 (1 at D = 64)
+                    uint32_t lo[32 * kHalfCh];
                     auto stage_chunk = [&](int c, const uint32_t *v) {
-                        uint8_t *line = (c < 2 ? sQ : sdO) + stage * kTileBytes + (c & 1) * 16384 + row * 128;
+                        uint8_t *line = (c < kHalfCh ? sQ : sdO) + stage * kTileBytes + (c % kHalfCh) * 16384 + row * 128;
 #pragma unroll
                         for (int ch = 0; ch < 8; ++ch)
                             *reinterpret_cast<uint4 *>(line + ((ch ^ (row & 7)) << 4)) =
@@ -307,14 +313,15 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     {
                         uint32_t hi[32];
 #pragma unroll
-                        for (int c = 2; c < 4; ++c) {
+                        for (int c = kHalfCh; c < kDqChunks; ++c) {
                             tmem_ld_x32(tmem + kColDP + 32 * c + lane_addr, hi);
                             tmem_wait_ld();
                             stage_chunk(c, hi);
                         }
                     }
-                    tmem_ld_x32(tmem + kColDP + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&lo[0]));
-                    tmem_ld_x32(tmem + kColDP + 32 + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&lo[32]));
+#pragma unroll
+                    for (int c = 0; c < kHalfCh; ++c)
+                        tmem_ld_x32(tmem + kColDP + 32 * c + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&lo[32 * c]));
                     tmem_wait_ld();
                     tc_fence_before();
                     __syncwarp();
@@ -322,18 +329,18 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     BPH_T(v2);
                     BWD_WAIT(&bars->qdo_mma_done[stage], ph, 14, m);     // product (4) has read the Q half
                     BPH_T(v3);
-                    stage_chunk(0, &lo[0]);
-                    stage_chunk(1, &lo[32]);
+#pragma unroll
+                    for (int c = 0; c < kHalfCh; ++c) stage_chunk(c, &lo[32 * c]);
                     fence_proxy_async_smem();
                     __syncwarp();
 #ifndef BWD_NO_RED
                     if (lane == 0) {
                         const int row0 = item.bl * p.S + m * kT + wq * 32;
 #pragma unroll
-                        for (int c = 0; c < 4; ++c)
+                        for (int c = 0; c < kDqChunks; ++c)
                             if (32 * c < p.Dg)          // a chunk wholly past the head dimension is padding
                             tma_reduce_add_3d(&p.dq_acc[item.r],
-                                              (c < 2 ? sQ : sdO) + stage * kTileBytes + (c & 1) * 16384 + wq * 4096,
+                                              (c < kHalfCh ? sQ : sdO) + stage * kTileBytes + (c % kHalfCh) * 16384 + wq * 4096,
                                               32 * c, h, row0);
                         tma_store_commit();
                         tma_store_wait_read<0>();          // these warps have nothing else to do until the next dQ tile
@@ -357,7 +364,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             if (lane == 0) {
                 mbar_arrive_expect_tx(&bars->kv_full, 2 * kTileBytes);
                 const int row0 = item.bl * p.S + item.n * kT;
-                for (int s = 0; s < 2; ++s) {
+                for (int s = 0; s < kSlabs; ++s) {
                     tma_load_3d(sK + s * 16384, &p.k[item.r], &bars->kv_full, s * 64, item.hkv, row0);
                     tma_load_3d(sV + s * 16384, &p.v[item.r], &bars->kv_full, s * 64, item.hkv, row0);
                 }
@@ -370,7 +377,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     if (lane == 0) {
                         mbar_arrive_expect_tx(&bars->qdo_full[stage], 2 * kTileBytes);
                         const int row0 = item.bl * p.S + m * kT;
-                        for (int s = 0; s < 2; ++s) {
+                        for (int s = 0; s < kSlabs; ++s) {
                             tma_load_3d(sQ + stage * kTileBytes + s * 16384, &p.q[item.r], &bars->qdo_full[stage], s * 64, h, row0);
                             tma_load_3d(sdO + stage * kTileBytes + s * 16384, &p.dout[item.r], &bars->qdo_full[stage], s * 64, h, row0);
                         }
@@ -594,9 +601,15 @@ int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, 
     BASP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const long long items = (long long)((pl->S + kT - 1) / kT) * pl->N * pl->Bl * pl->Hkv_l;
     const int grid = (int)(items < sms ? items : sms);
-    const int smem = 7 * kT * 128 * 2 + 4 * kT * (int)sizeof(float) + (int)sizeof(BwdBars);
-    BASP_CUDA_TRY(cudaFuncSetAttribute(attn_bwd_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    attn_bwd_kernel<R><<<grid, kBwdThreads, smem, st>>>(prm);
+    if (pl->D > 64) {        // 80 .. 128: the 128-wide kernel
+        const int smem = 6 * kT * 128 * 2 + 2 * 16384 + 4 * kT * (int)sizeof(float) + (int)sizeof(BwdBars);
+        BASP_CUDA_TRY(cudaFuncSetAttribute(attn_bwd_kernel<128, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attn_bwd_kernel<128, R><<<grid, kBwdThreads, smem, st>>>(prm);
+    } else {                 // 16 .. 64: half the tile bytes, half the accumulator columns, half the dQ reductions
+        const int smem = 6 * kT * 64 * 2 + 2 * 16384 + 4 * kT * (int)sizeof(float) + (int)sizeof(BwdBars);
+        BASP_CUDA_TRY(cudaFuncSetAttribute(attn_bwd_kernel<64, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attn_bwd_kernel<64, R><<<grid, kBwdThreads, smem, st>>>(prm);
+    }
     BASP_CUDA_TRY(cudaGetLastError());
 
     const long long n8 = (long long)(acc_b / sizeof(float) / 8);
