@@ -80,8 +80,9 @@ __device__ __forceinline__ bool bwd_get_item(const BwdParams<R> &p, int round, B
 }
 
 struct BwdBars {
-    uint64_t kv_full, kv_empty, qdo_full[2], qdo_empty[2], qdo_mma_done[2];
-    uint64_t s_full, stats_full[2], pds_ready, dq_full, dq_read, dkdv_full, dkdv_read;
+    uint64_t kv_full, kv_empty, qdo_full[3], qdo_empty[2], qdo_mma_done[3];      // (the 64-wide kernel has three stages)
+    uint64_t s_full, stats_full[3], pds_ready, dq_full, dq_read, dkdv_full, dkdv_read;
+    uint64_t s_full_b[2], dp_full;      // the pipelined 64-wide kernel: one S^T barrier per buffer, dP^T on its own
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -512,6 +513,8 @@ bwd_done:
     if (warp == kBwdTmaWarp) tmem_dealloc(tmem, 512);
 }
 
+#include "attn_bwd_d64.cuh"
+
 #undef BWD_WAIT
 
 // Delta[bl][h][s] = sum_d O[bl][s][h][d] * dO[bl][s][h][d]; one 16-lane group per (s, h) row of D <= 128.
@@ -605,10 +608,16 @@ int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, 
         const int smem = 6 * kT * 128 * 2 + 2 * 16384 + 4 * kT * (int)sizeof(float) + (int)sizeof(BwdBars);
         BASP_CUDA_TRY(cudaFuncSetAttribute(attn_bwd_kernel<128, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         attn_bwd_kernel<128, R><<<grid, kBwdThreads, smem, st>>>(prm);
-    } else {                 // 16 .. 64: half the tile bytes, half the accumulator columns, half the dQ reductions
+    } else {                 // 16 .. 64: the pipelined 64-wide kernel (attn_bwd_d64.cuh)
+#ifdef BASP_BWD64_PLAIN
         const int smem = 6 * kT * 64 * 2 + 2 * 16384 + 4 * kT * (int)sizeof(float) + (int)sizeof(BwdBars);
         BASP_CUDA_TRY(cudaFuncSetAttribute(attn_bwd_kernel<64, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         attn_bwd_kernel<64, R><<<grid, kBwdThreads, smem, st>>>(prm);
+#else
+        const int smem = (2 + 2 * 3) * kT * 64 * 2 + 4 * 16384 + 2 * 3 * kT * (int)sizeof(float) + (int)sizeof(BwdBars);
+        BASP_CUDA_TRY(cudaFuncSetAttribute(attn_bwd_d64_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attn_bwd_d64_kernel<R><<<grid, kBwdThreads, smem, st>>>(prm);
+#endif
     }
     BASP_CUDA_TRY(cudaGetLastError());
 
