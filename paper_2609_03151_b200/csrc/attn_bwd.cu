@@ -82,7 +82,7 @@ __device__ __forceinline__ bool bwd_get_item(const BwdParams<R> &p, int round, B
 struct BwdBars {
     uint64_t kv_full, kv_empty, qdo_full[3], qdo_empty[2], qdo_mma_done[3];      // (the 64-wide kernel has three stages)
     uint64_t s_full, stats_full[3], pds_ready, dq_full, dq_read, dkdv_full, dkdv_read;
-    uint64_t s_full_b[2], dp_full;      // the pipelined 64-wide kernel: one S^T barrier per buffer, dP^T on its own
+    uint64_t s_full_b[2], dp_full, p_ready;   // the pipelined 64-wide kernel: one S^T barrier per buffer, dP^T and P^T on their own
     uint32_t tmem_base;
     int abort_flag;
 };

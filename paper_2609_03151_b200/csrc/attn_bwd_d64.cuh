@@ -7,8 +7,9 @@
 //     the exponentials and the dS arithmetic;
 //   - a dQ staging buffer of its own, so a Q / dO stage is free for the next load as soon as the products that read it
 //     are done instead of after the reduce-add.
-// Per step the chain is then: P^T, dS^T ready -> dV, dQ, dK -> dP^T of the next step -> its dS arithmetic; the next
-// step's exponentials and the load and S^T product of the step after run underneath.
+//   - P^T as a hand-off of its own too: product (3) dV += P^T dO of a step is issued as soon as its P^T is in TMEM.
+// Per step the chain is then: dS^T ready -> dQ, dK -> dP^T of the next step -> its dS arithmetic; the next step's
+// exponentials, its dV product and the load and S^T product of the step after run underneath.
 // TMEM columns: S^T buffers at 0 and 128, dP^T / dQ at 256, dK at 384, dV at 448.
 #pragma once
 #ifdef BPH_ONLY_C
@@ -60,6 +61,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_d64_kernel(const __gr
         mbar_init(&bars->s_full_b[0], 1);
         mbar_init(&bars->s_full_b[1], 1);
         mbar_init(&bars->dp_full, 1);
+        mbar_init(&bars->p_ready, kBwdComputeWarps);
         mbar_init(&bars->pds_ready, kBwdComputeWarps);
         mbar_init(&bars->dq_full, 1);
         mbar_init(&bars->dq_read, 4);
@@ -136,6 +138,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_d64_kernel(const __gr
                             pk[c] = pack_bf16x2(__uint_as_float(st[2 * c]), __uint_as_float(st[2 * c + 1]));
                         tmem_st_x16(st_col, pk);
                     }
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->p_ready);          // product (3) of this step may start
                     // dS^T = P^T (dP^T scale - Delta scale): dP^T arrives after dQ of the step before has left TMEM
                     BPHC_T(t2);
                     BWD_WAIT(&bars->dp_full, it_g & 1, 12, m);
@@ -166,8 +172,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_d64_kernel(const __gr
                                 make_uint4(dp[4 * ch], dp[4 * ch + 1], dp[4 * ch + 2], dp[4 * ch + 3]);
                     }
                     fence_proxy_async_smem();
-                    tmem_wait_st();
-                    tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars->pds_ready);
                     BPHC_T(t4);
@@ -351,24 +355,35 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_d64_kernel(const __gr
                 }
                 return true;
             };
+            // (3) dV += P^T dO of step `it`, as soon as its P^T is in TMEM: A = P^T in the step's S^T buffer, B = dO read
+            //     MN-major.  The first one of an item also waits until dK / dV of the item before have been stored.
+            auto issue_dv = [&](uint32_t it, bool first) -> bool {
+                const uint32_t stage = it % kQS, buf = it & 1;
+                if (!mbar_wait(&bars->p_ready, it & 1, &bars->abort_flag)) return false;
+                if (first && !mbar_wait(&bars->dkdv_read, (item_n & 1) ^ 1, &bars->abort_flag)) return false;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t do16 = adO + stage * (kTileBytes >> 4);
+#pragma unroll
+                    for (int kk = 0; kk < kT / 16; ++kk)
+                        mma_ts(tmem + kColDV, tmem + kColST + 128 * buf + (kk / 2) * 32 + (kk % 2) * 8,
+                               desc_mn | (uint64_t)(do16 + kk * 128), idesc_kn, kk > 0 ? 1u : (first ? 0u : 1u));
+                }
+                return true;
+            };
             bool ok = issue_s(it_g) && issue_dp(it_g);
             if (ok && steps > 1) ok = issue_s(it_g + 1);
+            if (ok) ok = issue_dv(it_g, true);
             if (!ok) { bars->abort_flag = 1; bwd_report(p.status, 3, 31, item.n); goto bwd_done; }
             for (uint32_t j = 0; j < steps; ++j) {
-                const uint32_t it = it_g + j, stage = it % kQS, buf = it & 1;
-                const uint32_t q16 = aQ + stage * (kTileBytes >> 4), do16 = adO + stage * (kTileBytes >> 4);
+                const uint32_t it = it_g + j, stage = it % kQS;
+                const uint32_t q16 = aQ + stage * (kTileBytes >> 4);
                 BPHM_T(u0);
                 BWD_WAIT(&bars->pds_ready, it & 1, 33, (int)j);
-                if (j == 0) BWD_WAIT(&bars->dkdv_read, (item_n & 1) ^ 1, 34, item.n);
                 tc_fence_after();
                 BPHM_T(u1);
                 if (lane == 0) {
                     const uint32_t acc0 = j == 0 ? 0u : 1u;
-                    // (3) dV += P^T dO : A = P^T in the step's S^T buffer, B = dO read MN-major
-#pragma unroll
-                    for (int kk = 0; kk < kT / 16; ++kk)
-                        mma_ts(tmem + kColDV, tmem + kColST + 128 * buf + (kk / 2) * 32 + (kk % 2) * 8,
-                               desc_mn | (uint64_t)(do16 + kk * 128), idesc_kn, kk > 0 ? 1u : acc0);
                     // (5) dQ_m = dS K : A = the dS^T buffer read MN-major (query rows), B = K MN-major
 #pragma unroll
                     for (int kk = 0; kk < kT / 16; ++kk)
@@ -382,11 +397,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_d64_kernel(const __gr
                         mma_ss(tmem + kColDK, desc_k | (uint64_t)(adS + off), desc_mn | (uint64_t)(q16 + kk * 128),
                                idesc_kn, kk > 0 ? 1u : acc0);
                     }
-                    tc_commit(&bars->qdo_mma_done[stage]);        // the stage may be loaded again
+                    tc_commit(&bars->qdo_mma_done[stage]);        // (3), issued a step ago, and (4) are done: the stage may be loaded again
                 }
                 BPHM_T(u2);
                 ok = true;
-                if (j + 1 < steps) ok = issue_dp(it + 1);
+                if (j + 1 < steps) ok = issue_dp(it + 1) && issue_dv(it + 1, false);
                 BPHM_T(u3);
                 if (ok && j + 2 < steps) ok = issue_s(it + 2);
                 BPHM_T(u4);
