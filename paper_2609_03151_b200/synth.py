@@ -68,6 +68,9 @@ WORKLOADS = {
 for _b in (1, 2, 4, 8):
     WORKLOADS[f"e5_b{_b}_basp"] = Workload(f"e5_b{_b}_basp", N=8, B=_b, S=8192, Hq=32, Hkv=8, D=64)
     WORKLOADS[f"e5_b{_b}_ulysses"] = Workload(f"e5_b{_b}_ulysses", N=8, B=_b, S=8192, Hq=32, Hkv=8, D=64, G=1)
+# the same model shape as a training step (forward + backward), at the sweep's centre and at a long sequence
+WORKLOADS["e5_b2_train"] = Workload("e5_b2_train", N=8, B=2, S=8192, Hq=32, Hkv=8, D=64, train=True)
+WORKLOADS["llama32_1b_64k_train"] = Workload("llama32_1b_64k_train", N=8, B=1, S=65536, Hq=32, Hkv=8, D=64, train=True)
 for _s in (1, 2, 4, 8, 16, 32):
     WORKLOADS[f"e6_s{_s}k_basp"] = Workload(f"e6_s{_s}k_basp", N=8, B=2, S=_s * 1024, Hq=24, Hkv=8, D=128)
     WORKLOADS[f"e6_s{_s}k_ulysses"] = Workload(f"e6_s{_s}k_ulysses", N=8, B=2, S=_s * 1024, Hq=24, Hkv=8, D=128, G=1)
