@@ -260,6 +260,15 @@ int basp_attn_bwd(const basp_plan *plan, const void *const *q_head, const void *
                   void *const *dv_head, void *workspace, size_t workspace_bytes, float softmax_scale,
                   void *stream);
 size_t basp_attn_bwd_workspace_bytes(const basp_plan *plan);
+/* The same gradients, bit-identical from run to run: two passes (dK and dV with the key tile resident, dQ with the
+ * query tile resident) instead of one pass that adds dQ partial sums into a global accumulator in whatever order the
+ * thread blocks finish.  Costs the scores and the element-wise part twice (measured about 7 % slower on the config 5
+ * shape); same arguments, workspace and errors as basp_attn_bwd. */
+int basp_attn_bwd_deterministic(const basp_plan *plan, const void *const *q_head, const void *const *k_head,
+                                const void *const *v_head, const void *const *o_head, const void *const *do_head,
+                                const float *const *lse_shards, void *const *dq_head, void *const *dk_head,
+                                void *const *dv_head, void *workspace, size_t workspace_bytes, float softmax_scale,
+                                void *stream);
 
 /* dQ (Hq heads), dK and dV (Hkv heads) head- to sequence-sharded in ONE launch: the reverse
  * all-to-alls of the gradients. */

@@ -31,7 +31,7 @@ EXPORTS = [
     "basp_layer_bwd", "basp_layer_bwd_workspace_bytes", "basp_get_status", "basp_clear_status",
     "basp_strerror", "basp_last_cuda_error", "basp_launch_count", "basp_selftest_wait_timeout", "basp_qkv_proj", "basp_out_proj",
     "basp_reshard_qkv_s2h_ranks", "basp_reshard_h2s_ranks", "basp_attn_fwd_ranks", "basp_layer_fwd_fused_ranks",
-    "basp_qkv_proj_rope", "basp_layer_bwd_seq", "basp_layer_bwd_seq_workspace_bytes", "basp_plan_create_parts",
+    "basp_qkv_proj_rope", "basp_layer_bwd_seq", "basp_layer_bwd_seq_workspace_bytes", "basp_plan_create_parts", "basp_attn_bwd_deterministic",
 ]
 
 
@@ -71,6 +71,7 @@ lib.basp_layer_fwd_static.argtypes = [c_void_p] + [_PP] * 5 + [c_float, c_void_p
 lib.basp_layer_fwd_host.argtypes = [c_void_p] + [_PP] * 4 + [c_void_p, c_size_t, c_float, c_void_p]
 lib.basp_layer_workspace_shards.argtypes = [c_void_p, c_void_p] + [_PP] * 4
 lib.basp_attn_bwd.argtypes = [c_void_p] + [_PP] * 9 + [c_void_p, c_size_t, c_float, c_void_p]
+lib.basp_attn_bwd_deterministic.argtypes = lib.basp_attn_bwd.argtypes
 lib.basp_reshard_grads_h2s.argtypes = [c_void_p] + [_PP] * 6 + [c_void_p]
 lib.basp_layer_bwd.argtypes = [c_void_p] + [_PP] * 9 + [c_void_p, c_size_t, c_float, c_void_p]
 lib.basp_layer_bwd_seq.argtypes = [c_void_p] + [_PP] * 9 + [c_void_p, c_size_t, c_float, c_void_p]
@@ -335,9 +336,10 @@ def basp_layer_bwd_workspace_bytes(plan) -> int:
 
 
 def basp_attn_bwd(plan, q_head, k_head, v_head, o_head, do_head, lse_shards, dq_head, dk_head, dv_head, workspace,
-                  softmax_scale=0.0, stream=None):
+                  softmax_scale=0.0, stream=None, deterministic=False):
     n = plan.N
-    _check(lib.basp_attn_bwd(plan.handle, *[_ptrs(t, n) for t in (q_head, k_head, v_head, o_head, do_head, lse_shards,
+    fn = lib.basp_attn_bwd_deterministic if deterministic else lib.basp_attn_bwd
+    _check(fn(plan.handle, *[_ptrs(t, n) for t in (q_head, k_head, v_head, o_head, do_head, lse_shards,
                                                                   dq_head, dk_head, dv_head)],
                              c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size(),
                              softmax_scale, _stream(stream)), "basp_attn_bwd")

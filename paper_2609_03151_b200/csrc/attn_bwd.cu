@@ -49,6 +49,7 @@ struct BwdParams {
     const float *lse[R];
     const float *delta[R];
     __nv_bfloat16 *dk[R], *dv[R];
+    __nv_bfloat16 *dq[R];       // the two-pass kernels write dQ directly
     int n_ranks, Bl, S, Hq_l, Hkv_l, q_per_kv, causal;
     int Dg;                     // head dimension in memory (a multiple of 16 up to 128): the tile loads zero-fill the columns
                                 // past it, so every product is right as it stands; only the stores have to skip them
@@ -514,6 +515,7 @@ bwd_done:
 }
 
 #include "attn_bwd_d64.cuh"
+#include "attn_bwd_2pass.cuh"
 
 #undef BWD_WAIT
 
@@ -562,7 +564,7 @@ size_t bwd_delta_bytes(const basp_plan *p) { return (((size_t)p->Bl * p->Hq_l * 
 template <int R>
 int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, const void *const *v,
                const void *const *o, const void *const *dout, const float *const *lse, void *const *dq,
-               void *const *dk, void *const *dv, char *ws, float scale, cudaStream_t st) {
+               void *const *dk, void *const *dv, char *ws, float scale, bool two_pass, cudaStream_t st) {
     BwdParams<R> prm;
     const uint64_t rows = (uint64_t)pl->Bl * pl->S;
     const size_t acc_b = bwd_acc_bytes(pl), del_b = bwd_delta_bytes(pl);
@@ -580,6 +582,7 @@ int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, 
         if (rc != BASP_OK) return rc;
         prm.delta[r] = reinterpret_cast<float *>(reinterpret_cast<char *>(del0) + (size_t)r * del_b);
         prm.dk[r] = (__nv_bfloat16 *)dk[r];
+        prm.dq[r] = (__nv_bfloat16 *)dq[r];
         prm.dv[r] = (__nv_bfloat16 *)dv[r];
     }
     prm.n_ranks = pl->N; prm.Bl = pl->Bl; prm.S = pl->S; prm.Hq_l = pl->Hq_l; prm.Hkv_l = pl->Hkv_l;
@@ -590,7 +593,7 @@ int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, 
     prm.status = basp_status_device_ptr();
     if (!prm.status) return BASP_ERR_CUDA;
 
-    BASP_CUDA_TRY(cudaMemsetAsync(acc0, 0, (size_t)pl->N * acc_b, st));
+    if (!two_pass) BASP_CUDA_TRY(cudaMemsetAsync(acc0, 0, (size_t)pl->N * acc_b, st));
     const long long row_threads = (long long)pl->Bl * pl->S * pl->Hq_l * 16;
     for (int r = 0; r < pl->N; ++r) {
         bwd_delta_kernel<<<(unsigned)((row_threads + 255) / 256), 256, 0, st>>>(
@@ -602,8 +605,20 @@ int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, 
     int dev = 0, sms = 0;
     BASP_CUDA_TRY(cudaGetDevice(&dev));
     BASP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    const long long items = (long long)((pl->S + kT - 1) / kT) * pl->N * pl->Bl * pl->Hkv_l;
+    const long long n_tiles = (pl->S + kT - 1) / kT;
+    const long long items = n_tiles * pl->N * pl->Bl * pl->Hkv_l;
     const int grid = (int)(items < sms ? items : sms);
+    if (two_pass) {
+        const int smem = 6 * kT * 128 * 2 + 2 * 16384 + 4 * kT * (int)sizeof(float) + (int)sizeof(BwdBars);
+        BASP_CUDA_TRY(cudaFuncSetAttribute(attn_bwd_pass_kernel<0, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        BASP_CUDA_TRY(cudaFuncSetAttribute(attn_bwd_pass_kernel<1, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attn_bwd_pass_kernel<0, R><<<grid, kBwdThreads, smem, st>>>(prm);
+        const long long items_q = n_tiles * pl->N * pl->Bl * pl->Hq_l;
+        attn_bwd_pass_kernel<1, R><<<(int)(items_q < sms ? items_q : sms), kBwdThreads, smem, st>>>(prm);
+        BASP_CUDA_TRY(cudaGetLastError());
+        basp_count_launch(2 + pl->N);
+        return BASP_OK;
+    }
     if (pl->D > 64) {        // 80 .. 128: the 128-wide kernel
         const int smem = 6 * kT * 128 * 2 + 2 * 16384 + 4 * kT * (int)sizeof(float) + (int)sizeof(BwdBars);
         BASP_CUDA_TRY(cudaFuncSetAttribute(attn_bwd_kernel<128, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
@@ -645,11 +660,12 @@ extern "C" size_t basp_attn_bwd_workspace_bytes(const basp_plan *p) {
     return (size_t)p->N * (bwd_acc_bytes(p) + bwd_delta_bytes(p));
 }
 
-extern "C" int basp_attn_bwd(const basp_plan *pl, const void *const *q_head, const void *const *k_head,
-                             const void *const *v_head, const void *const *o_head, const void *const *do_head,
-                             const float *const *lse_shards, void *const *dq_head, void *const *dk_head,
-                             void *const *dv_head, void *workspace, size_t workspace_bytes, float softmax_scale,
-                             void *stream) {
+namespace {
+int bwd_entry(const basp_plan *pl, const void *const *q_head, const void *const *k_head,
+              const void *const *v_head, const void *const *o_head, const void *const *do_head,
+              const float *const *lse_shards, void *const *dq_head, void *const *dk_head,
+              void *const *dv_head, void *workspace, size_t workspace_bytes, float softmax_scale, bool two_pass,
+              void *stream) {
     if (!pl || !q_head || !k_head || !v_head || !o_head || !do_head || !lse_shards || !dq_head || !dk_head ||
         !dv_head || !workspace)
         return BASP_ERR_NULL;
@@ -671,7 +687,29 @@ extern "C" int basp_attn_bwd(const basp_plan *pl, const void *const *q_head, con
     }
     if (pl->N <= 8)
         return bwd_launch<8>(pl, q_head, k_head, v_head, o_head, do_head, lse_shards, dq_head, dk_head, dv_head,
-                             (char *)workspace, softmax_scale, (cudaStream_t)stream);
+                             (char *)workspace, softmax_scale, two_pass, (cudaStream_t)stream);
     return bwd_launch<BASP_MAX_RANKS>(pl, q_head, k_head, v_head, o_head, do_head, lse_shards, dq_head, dk_head,
-                                      dv_head, (char *)workspace, softmax_scale, (cudaStream_t)stream);
+                                      dv_head, (char *)workspace, softmax_scale, two_pass, (cudaStream_t)stream);
+}
+}  // namespace
+
+extern "C" int basp_attn_bwd(const basp_plan *pl, const void *const *q_head, const void *const *k_head,
+                             const void *const *v_head, const void *const *o_head, const void *const *do_head,
+                             const float *const *lse_shards, void *const *dq_head, void *const *dk_head,
+                             void *const *dv_head, void *workspace, size_t workspace_bytes, float softmax_scale,
+                             void *stream) {
+    return bwd_entry(pl, q_head, k_head, v_head, o_head, do_head, lse_shards, dq_head, dk_head, dv_head, workspace,
+                     workspace_bytes, softmax_scale, false, stream);
+}
+
+// The same gradients from the two-pass kernels (attn_bwd_2pass.cuh): no reduction through global memory, so the
+// result does not depend on the order in which CTAs finish (bit-identical from run to run), at 7 products per tile
+// pair instead of 5.
+extern "C" int basp_attn_bwd_deterministic(const basp_plan *pl, const void *const *q_head, const void *const *k_head,
+                                           const void *const *v_head, const void *const *o_head,
+                                           const void *const *do_head, const float *const *lse_shards,
+                                           void *const *dq_head, void *const *dk_head, void *const *dv_head,
+                                           void *workspace, size_t workspace_bytes, float softmax_scale, void *stream) {
+    return bwd_entry(pl, q_head, k_head, v_head, o_head, do_head, lse_shards, dq_head, dk_head, dv_head, workspace,
+                     workspace_bytes, softmax_scale, true, stream);
 }

@@ -28,7 +28,7 @@ def inputs(w, seed=0):
     return [synth.bits(t) for t in (q, k, v, do)], oracle.plan(w.N, w.B, w.S, w.G)
 
 
-def run_attn_bwd(basp, w, causal=True, seed=0):
+def run_attn_bwd(basp, w, causal=True, seed=0, deterministic=False):
     (Xq, Xk, Xv, Xdo), op = inputs(w, seed)
     pl = make_plan(basp, w, causal)
     qh, kh, vh, doh = (oracle.s2h(oracle.partition(X, op), op) for X in (Xq, Xk, Xv, Xdo))
@@ -41,8 +41,14 @@ def run_attn_bwd(basp, w, causal=True, seed=0):
     gk = [torch.full_like(t, float("nan")) for t in dk_]
     gv = [torch.full_like(t, float("nan")) for t in dk_]
     ws = torch.empty(basp.basp_attn_bwd_workspace_bytes(pl), dtype=torch.uint8, device="cuda")
-    basp.basp_attn_bwd(pl, dq_, dk_, dv_, o, ddo, lse, gq, gk, gv, ws)
+    basp.basp_attn_bwd(pl, dq_, dk_, dv_, o, ddo, lse, gq, gk, gv, ws, deterministic=deterministic)
     basp.basp_get_status()
+    if deterministic:      # the two-pass kernels add nothing up across thread blocks: a second run gives the same bits
+        again = [[torch.full_like(t, float("nan")) for t in x] for x in (gq, gk, gv)]
+        basp.basp_attn_bwd(pl, dq_, dk_, dv_, o, ddo, lse, again[0], again[1], again[2], ws, deterministic=True)
+        basp.basp_get_status()
+        for first, second in zip((gq, gk, gv), again):
+            assert all(torch.equal(a.view(torch.int16), b.view(torch.int16)) for a, b in zip(first, second))
     ref = [oracle.attn_bwd(qh[r], kh[r], vh[r], doh[r], causal=causal) for r in range(w.N)]
     return (to_f64(gq), to_f64(gk), to_f64(gv)), tuple(np.stack([g[n] for g in ref]) for n in ("dQ", "dK", "dV"))
 
@@ -58,19 +64,21 @@ def run_attn_bwd(basp, w, causal=True, seed=0):
     ("head_dim_80", synth.shrink(synth.WORKLOADS["t2_qwen25_3b"], 128)),                    # hidden 2560 / 32 heads
     ("head_dim_48", synth.Workload("d48", N=2, B=2, S=256, Hq=2, Hkv=1, D=48)),
 ])
-def test_attn_bwd_matches_oracle(basp, name, w):
-    got, ref = run_attn_bwd(basp, w)
+@pytest.mark.parametrize("deterministic", [False, True])
+def test_attn_bwd_matches_oracle(basp, name, w, deterministic):
+    got, ref = run_attn_bwd(basp, w, deterministic=deterministic)
     for g, r, n in zip(got, ref, ("dQ", "dK", "dV")):
         assert np.isfinite(g).all(), f"{name} {n}: not fully written"
         assert_grad_close(g, r, f"{name} {n}")
 
 
+@pytest.mark.parametrize("deterministic", [False, True])
 @pytest.mark.parametrize("S,causal", [(200, True), (333, True), (1000, True), (77, False), (129, True)])
-def test_attn_bwd_ragged_sequence_lengths(basp, S, causal):
+def test_attn_bwd_ragged_sequence_lengths(basp, S, causal, deterministic):
     """S not a multiple of the 128-row tile, two sequences per rank: what follows a ragged end is the next sequence (its
     rows must neither be read into the gradients nor be written), and the LSE / Delta rows are not 16-byte aligned."""
     w = synth.Workload("ragged_S", N=2, B=4, S=S, Hq=4, Hkv=2, D=128, G=2)
-    got, ref = run_attn_bwd(basp, w, causal=causal, seed=S)
+    got, ref = run_attn_bwd(basp, w, causal=causal, seed=S, deterministic=deterministic)
     for g, r, n in zip(got, ref, ("dQ", "dK", "dV")):
         assert np.isfinite(g).all(), f"S={S} {n}: not fully written"
         assert_grad_close(g, r, f"S={S} {n}")
