@@ -239,6 +239,7 @@ def run_gpu(args, w: synth.Workload):
     pdist.barrier()
     launches = basp.basp_launch_count() - launches0
     total_ms = ev[0][0].elapsed_time(ev[-1][n_ev - 1])
+    per_step = [e[0].elapsed_time(e[n_ev - 1]) for e in ev]          # each step on its own (the headline is total / steps)
     ms_s2h = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
     ms_attn = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
     ms_h2s = statistics.mean(e[2].elapsed_time(e[3]) for e in ev)
@@ -374,6 +375,7 @@ def run_gpu(args, w: synth.Workload):
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
                     "call": "basp_layer_fwd_host (fused kernel per arrived piece of query rows, copies and kernels pipelined, pinned host shards)"},
             "gpu_launches": launches,
+            "ms_per_step_median": statistics.median(per_step), "ms_per_step_best": min(per_step),
             "roofline": {"kernel": "attn_fwd", "bound": "tensor", "achieved": attn_tflops,
                          "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
                          "frac": attn_tflops / peaks["bf16_sustained"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
