@@ -142,3 +142,39 @@ def test_full_size_sampled_rows(basp, name):
         basp.basp_get_status()
         got = np.stack([do[b * K + i // T][0, i % T, h].float().cpu().numpy().astype(np.float64) for b, h, i in rows])
         assert_attn_close(got, ref, f"{name} fused={fused}")
+
+
+@pytest.mark.parametrize("scale", [0.0, 0.05])
+def test_four_sequences_per_group_and_custom_scale_forward_and_backward(basp, scale):
+    """Bl = 4 sequences per group (K = 2) with a caller-supplied softmax scale, through the forward layer (both forms)
+    and the backward layer; scale = 0 selects 1/sqrt(D)."""
+    w = synth.Workload("bl4", N=4, B=8, S=512, Hq=4, Hkv=2, D=128, G=2)
+    q, k, v, do_ = synth.make_qkv(w, seed=8, with_dO=True)
+    Xq, Xk, Xv, Xdo = (synth.bits(t) for t in (q, k, v, do_))
+    op = oracle.plan(w.N, w.B, w.S, w.G)
+    osc = None if scale == 0.0 else scale
+    ref = oracle.layer_fwd(Xq, Xk, Xv, op, scale=osc)
+    refb = oracle.layer_bwd(Xq, Xk, Xv, Xdo, op, scale=osc)
+    pl = make_plan(basp, w)
+    assert pl.Bl == 4 and pl.K == 2
+    dq, dk, dv, ddo = (to_dev(oracle.partition(X, op)) for X in (Xq, Xk, Xv, Xdo))
+    lse = [torch.zeros((pl.Bl, pl.Hq_l, pl.S), dtype=torch.float32, device="cuda") for _ in range(w.N)]
+    ws = torch.empty(basp.basp_workspace_bytes(pl), dtype=torch.uint8, device="cuda")
+    basp.basp_clear_status()
+    for fused in (True, False):
+        o = [torch.full_like(t, float("nan")) for t in dq]
+        if fused:
+            basp.basp_layer_fwd_fused(pl, dq, dk, dv, o, lse, softmax_scale=scale)
+        else:
+            basp.basp_layer_fwd(pl, dq, dk, dv, o, ws, lse_shards=lse, softmax_scale=scale)
+        basp.basp_get_status()
+        assert_attn_close(to_f64(o), ref["o_seq"], f"bl4 fused={fused} scale={scale}")
+    qh, kh, vh, oh = basp.basp_layer_workspace_shards(pl, ws)
+    gq, gk, gv = ([torch.full_like(t, float("nan")) for t in x] for x in (dq, dk, dv))
+    ws2 = torch.empty(basp.basp_layer_bwd_workspace_bytes(pl), dtype=torch.uint8, device="cuda")
+    basp.basp_layer_bwd(pl, qh, kh, vh, oh, lse, ddo, gq, gk, gv, ws2, softmax_scale=scale)
+    basp.basp_get_status()
+    for name, got in (("dq", gq), ("dk", gk), ("dv", gv)):
+        r = refb[name + "_seq"]
+        err = np.abs(to_f64(got) - r)
+        assert (err <= 2e-2 + 2.0 ** -8 * np.abs(r)).all(), (name, float(err.max()))
