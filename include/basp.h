@@ -220,7 +220,7 @@ int basp_layer_fwd_fused(const basp_plan *plan, const void *const *q_seq, const 
  *   basp_attn_fwd_ranks         attention over their own head shards (local memory only);
  *   basp_reshard_h2s_ranks      pulls their sequence shards of O together from the group's head shards (plain loads);
  *   basp_layer_fwd_fused_ranks  the three steps as one kernel: Q/K/V tiles are fetched from the group's sequence
- *                               shards wherever they live (TMA tile loads without multicast) and O tiles are stored
+ *                               shards wherever they live (plain TMA tile loads, one per thread block) and O tiles are stored
  *                               into the owner's sequence shard - exchange and attention overlap tile by tile.
  * The caller orders the GPUs on the host: every GPU's inputs are complete before any GPU launches, and nobody reuses
  * a buffer before all GPUs' launches have finished (a barrier of the process group on both sides; the kernels never

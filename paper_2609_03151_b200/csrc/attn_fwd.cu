@@ -153,7 +153,7 @@ extern "C" int basp_layer_fwd_fused(const basp_plan *plan, const void *const *q_
 // One physical GPU's share when the N ranks are spread over several GPUs: only ranks [rank_begin, rank_begin +
 // rank_count) compute.  Head-sharded operands of other ranks are not touched.  With sequence-sharded operands (fused)
 // the tiles of the other members of the range's groups are fetched from wherever their pointers lead - peer memory
-// mapped into this process included (plain TMA tile loads, no multicast) - and O tiles are stored there with plain
+// mapped into this process included (plain TMA tile loads, every CTA fetching its own tile) - and O tiles are stored there with plain
 // stores: the all-to-alls of Section IV-C and the attention in one kernel over NVLink.
 extern "C" int basp_attn_fwd_ranks(const basp_plan *plan, const void *const *q_head, const void *const *k_head,
                                    const void *const *v_head, void *const *o_head, float *const *lse_shards,

@@ -7,7 +7,7 @@ for weak scaling, different micro-batches -- and only timing is reduced across r
 When a group does span GPUs (K > N / world) the exchange is real: every GPU then runs the
 `*_ranks` calls for the ranks it hosts over shard tables that point into its peers' memory
 (`SymmetricShards`, `layer_fwd_fused_multi_gpu`); the kernels use plain loads/stores and TMA tile
-loads without multicast on that memory and never wait for one another.
+loads on that memory (every thread block fetches its own tile) and never wait for one another.
 """
 from __future__ import annotations
 
