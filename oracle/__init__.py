@@ -392,6 +392,22 @@ def attn_bwd_dkdv_tail(Q, K, V, dO, b: int, kv: int, ncols: int, scale: float | 
     return dK, dV
 
 
+def attn_bwd_dkdv_cols(Q, K, V, dO, b: int, kv: int, cols, scale: float | None = None, causal: bool = True):
+    """dK, dV of the key positions ``cols`` (any positions) of (sequence b, KV head kv) -> two [len(cols), D] fp64.
+    The row statistics (LSE, Delta) of every row that sees the smallest sampled column are formed once, from each
+    row's own definition, and shared by the columns."""
+    Q, K, V, dO = (np.ascontiguousarray(a, dtype=np.uint16) for a in (Q, K, V, dO))
+    cols = np.ascontiguousarray(cols, dtype=np.int32).reshape(-1)
+    Bn, S, Hq, D = Q.shape
+    assert 0 <= b < Bn and 0 <= kv < K.shape[2] and ((cols >= 0) & (cols < S)).all()
+    dK = np.empty((cols.shape[0], D), dtype=np.float64)
+    dV = np.empty((cols.shape[0], D), dtype=np.float64)
+    _load().oracle_attn_bwd_dkdv_cols(_p(Q), _p(K), _p(V), _p(dO), int(b), int(kv), _p(cols), int(cols.shape[0]),
+                                      _p(dK), _p(dV), S, Hq, K.shape[2], D, ctypes.c_double(_scale(scale, D)),
+                                      int(causal))
+    return dK, dV
+
+
 def layer_bwd(Xq, Xk, Xv, XdO, pl: Plan, scale: float | None = None, causal: bool = True):
     """Backward of the sequence-parallel layer, step by step: partition the four global tensors,
     all-to-all each to head-sharded, per-rank attention backward, reverse all-to-all of dQ, dK, dV,

@@ -420,3 +420,65 @@ void oracle_attn_bwd_dkdv_tail(const uint16_t *Q, const uint16_t *Kt, const uint
     free(lse);
     free(delta);
 }
+
+/* dK and dV of ARBITRARY key columns cols[0..ncols) of (sequence b, KV head kv).  Column j is summed over every row
+ * i that sees it (i >= j under the causal mask, all rows otherwise) of the Hq/Hkv query heads that read the KV head, so
+ * the row statistics LSE_i and D_i are needed for all rows from the smallest sampled column on: one pass over those
+ * rows (each from its own definition, O(i D) per row), shared by all sampled columns, then the column sums written
+ * out as in the full backward.  dK_cols, dV_cols [ncols][D]. */
+void oracle_attn_bwd_dkdv_cols(const uint16_t *Q, const uint16_t *Kt, const uint16_t *V, const uint16_t *dO,
+                               int b, int kv, const int *cols, int ncols, double *dK_cols, double *dV_cols, int S,
+                               int Hq, int Hkv, int D, double scale, int causal) {
+    const int rep = Hq / Hkv;
+    int i0 = 0;
+    if (causal) {
+        i0 = S;
+        for (int c = 0; c < ncols; ++c)
+            if (cols[c] < i0) i0 = cols[c];
+    }
+    const int nrows = S - i0;
+    if (ncols <= 0 || nrows <= 0) return;
+    double *lse = (double *)malloc(sizeof(double) * (size_t)rep * nrows);
+    double *delta = (double *)malloc(sizeof(double) * (size_t)rep * nrows);
+#pragma omp parallel
+    {
+        double *scores = (double *)malloc(sizeof(double) * (size_t)S);
+        double *o_row = (double *)malloc(sizeof(double) * (size_t)D);
+#pragma omp for schedule(dynamic, 4)
+        for (long r = 0; r < (long)rep * nrows; ++r) {
+            const long rr = (long)rep * nrows - 1 - r;          /* long rows first; the order is irrelevant */
+            const int hh = (int)(rr / nrows), i = i0 + (int)(rr % nrows);
+            bwd_row_stats(Q, Kt, V, dO, S, Hq, Hkv, D, scale, causal, b, kv * rep + hh, i, scores, o_row,
+                          &lse[(size_t)hh * nrows + (i - i0)], &delta[(size_t)hh * nrows + (i - i0)]);
+        }
+        free(scores);
+        free(o_row);
+    }
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int c = 0; c < ncols; ++c) {
+        const int j = cols[c];
+        const uint16_t *k = Kt + (((size_t)b * S + j) * Hkv + kv) * D;
+        const uint16_t *v = V + (((size_t)b * S + j) * Hkv + kv) * D;
+        double *dk_row = dK_cols + (size_t)c * D, *dv_row = dV_cols + (size_t)c * D;
+        for (int d = 0; d < D; ++d) dk_row[d] = dv_row[d] = 0.0;
+        for (int hh = 0; hh < rep; ++hh)
+            for (int i = causal ? j : 0; i < S; ++i) {
+                const int h = kv * rep + hh;
+                const uint16_t *q = Q + (((size_t)b * S + i) * Hq + h) * D;
+                const uint16_t *go = dO + (((size_t)b * S + i) * Hq + h) * D;
+                double s = 0.0, dp = 0.0;
+                for (int d = 0; d < D; ++d) {
+                    s += bf16_to_f64(q[d]) * bf16_to_f64(k[d]);
+                    dp += bf16_to_f64(go[d]) * bf16_to_f64(v[d]);
+                }
+                const double p = exp(s * scale - lse[(size_t)hh * nrows + (i - i0)]);
+                const double ds = p * (dp - delta[(size_t)hh * nrows + (i - i0)]);
+                for (int d = 0; d < D; ++d) {
+                    dv_row[d] += p * bf16_to_f64(go[d]);
+                    dk_row[d] += scale * ds * bf16_to_f64(q[d]);
+                }
+            }
+    }
+    free(lse);
+    free(delta);
+}

@@ -99,6 +99,26 @@ def test_sparse_entries_match_full():
     assert np.allclose(dv, g["dV"][1, S - 7:, 1], rtol=0, atol=1e-13)
 
 
+@pytest.mark.parametrize("causal", [True, False])
+def test_column_entry_matches_library_autograd_and_full_entry(causal):
+    """The arbitrary-column dK/dV entry (used for the large shapes): unordered columns, a repeated one, the first and
+    the last position, on a GQA shape; against fp64 autograd of the library routine and against the full entry."""
+    Bn, S, Hq, Hkv, D = 2, 61, 6, 2, 8
+    Q, K, V, dO = (rand_bits(s, 50 + i) for i, s in enumerate([(Bn, S, Hq, D), (Bn, S, Hkv, D), (Bn, S, Hkv, D), (Bn, S, Hq, D)]))
+    _, rk, rv = autograd_ref(Q, K, V, dO, 0.3, causal)
+    g = oracle.attn_bwd(Q, K, V, dO, scale=0.3, causal=causal)
+    cols = [40, 7, 60, 0, 7, 33]
+    for b, kv in ((0, 0), (1, 1)):
+        dk, dv = oracle.attn_bwd_dkdv_cols(Q, K, V, dO, b=b, kv=kv, cols=cols, scale=0.3, causal=causal)
+        assert np.abs(dk - rk[b, cols, kv]).max() < 1e-11
+        assert np.abs(dv - rv[b, cols, kv]).max() < 1e-11
+        assert np.allclose(dk, g["dK"][b, cols, kv], rtol=0, atol=1e-13)
+        assert np.allclose(dv, g["dV"][b, cols, kv], rtol=0, atol=1e-13)
+    # a single late column needs the statistics of the rows behind it only, and gives the same numbers
+    dk1, dv1 = oracle.attn_bwd_dkdv_cols(Q, K, V, dO, b=1, kv=1, cols=[55], scale=0.3, causal=causal)
+    assert np.allclose(dk1[0], g["dK"][1, 55, 1], rtol=0, atol=1e-13) and np.allclose(dv1[0], g["dV"][1, 55, 1], rtol=0, atol=1e-13)
+
+
 def test_layer_bwd_grouping_equivalence():
     N, B, S, Hq, Hkv, D = 4, 2, 32, 8, 4, 4
     X = [rand_bits(s, 40 + i) for i, s in enumerate([(B, S, Hq, D), (B, S, Hkv, D), (B, S, Hkv, D), (B, S, Hq, D)])]
