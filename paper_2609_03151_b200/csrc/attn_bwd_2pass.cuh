@@ -39,9 +39,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_pass_kernel(const __g
 
     const int tid = threadIdx.x, warp = __shfl_sync(0xffffffffu, tid >> 5, 0), lane = tid & 31;
     const int n_t = (p.S + kT - 1) / kT;               // tiles per sequence (the last one may be ragged)
-#ifdef BASP_PHASE_TIMING
-    long long bacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-#endif
 
     // Work items, longest first.  Pass KV: low key tiles are seen by the most query tiles; pass Q: high query tiles see
     // the most key tiles.
@@ -127,11 +124,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_pass_kernel(const __g
                 int head, tile;
                 step_of(item, j, head, tile);
                 const int buf = it_g & 1;
-                BPH_T(t0);
                 if (kKV) BWD_WAIT(&bars->stats_full[buf], (it_g >> 1) & 1, 10, j);
                 BWD_WAIT(&bars->s_full, it_g & 1, 11, j);
                 tc_fence_after();
-                BPH_T(t1);
                 uint32_t st[32], dp[32];
                 tmem_ld_x32(tmem + kColST + 32 * g + lane_addr, st);
                 tmem_wait_ld();
@@ -191,10 +186,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_pass_kernel(const __g
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars->p_ready);
                 }
-                BPH_T(t2);
                 BWD_WAIT(&bars->dp_full, it_g & 1, 12, j);
                 tc_fence_after();
-                BPH_T(t3);
                 tmem_ld_x32(tmem + kColDP + 32 * g + lane_addr, dp);
                 tmem_wait_ld();
 #pragma unroll
@@ -224,8 +217,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_pass_kernel(const __g
                 tc_fence_before();          // the dP^T columns have been read: (2) of the next step may overwrite them
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars->pds_ready);
-                BPH_T(t4);
-                BPH_ADD(0, t0, t1); BPH_ADD(1, t1, t2); BPH_ADD(2, t2, t3); BPH_ADD(3, t3, t4); BPH_ADD(6, t0, t0 + 1);
             }
             // ---- item done: the accumulators to global memory as bf16
             BWD_WAIT(&bars->dkdv_full, item_n & 1, 13, item.t);
@@ -381,9 +372,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_pass_kernel(const __g
                 const uint32_t it = it_g + j, stage = it & 1;
                 const uint32_t y0 = aY0 + stage * (kTileBytes >> 4), y1 = aY1 + stage * (kTileBytes >> 4);
                 const uint32_t acc0 = j == 0 ? 0u : 1u;
-                BPH_T(u0);
                 BWD_WAIT(&bars->p_ready, it & 1, 32, (int)j);
-                BPH_T(u1);
                 if (j == 0) BWD_WAIT(&bars->dkdv_read, (item_n & 1) ^ 1, 34, item.t);   // the accumulators of the item before are stored
                 tc_fence_after();
                 if (kKV && lane == 0) {
@@ -395,10 +384,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_pass_kernel(const __g
                                desc_mn | (uint64_t)(y1 + kk * 128), idesc_kn, kk > 0 ? 1u : acc0);
                 }
                 if (j + 1 < steps && !issue_s(it + 1)) { bars->abort_flag = 1; bwd_report(p.status, 3, 35, (int)j); goto bwd_done; }
-                BPH_T(u2);
                 BWD_WAIT(&bars->pds_ready, it & 1, 33, (int)j);
                 tc_fence_after();
-                BPH_T(u3);
                 if (lane == 0) {
                     // (4) ACC0 += dS Y0 : A = dS from shared memory (K-major), B = Y0 read MN-major
 #pragma unroll
@@ -410,8 +397,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_pass_kernel(const __g
                     tc_commit(&bars->qdo_mma_done[stage]);        // (3) and (4) are done with the stage
                 }
                 if (j + 1 < steps) issue_dp(it + 1);
-                BPH_T(u4);
-                BPH_ADD(0, u0, u1); BPH_ADD(1, u1, u2); BPH_ADD(2, u2, u3); BPH_ADD(3, u3, u4); BPH_ADD(6, u0, u0 + 1);
             }
             it_g += steps;
             if (lane == 0) {
@@ -423,12 +408,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_pass_kernel(const __g
     }
 
 bwd_done:
-#ifdef BASP_PHASE_TIMING
-    if (blockIdx.x == 5 && (threadIdx.x & 31) == 0 && (warp == 0 || warp == kBwdMmaWarp)) {
-        const int base_ = (warp == 0 ? 0 : 8) + (kKV ? 0 : 16);
-        for (int i_ = 0; i_ < 8; ++i_) g_bwd_phase[base_ + i_] += bacc[i_];
-    }
-#endif
     tc_fence_before();
     __syncthreads();
     if (bars->abort_flag) {

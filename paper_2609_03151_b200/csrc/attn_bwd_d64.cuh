@@ -30,9 +30,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_d64_kernel(const __gr
     BwdBars *bars = reinterpret_cast<BwdBars *>(s_delta + kQS * kT);
 
     const int tid = threadIdx.x, warp = __shfl_sync(0xffffffffu, tid >> 5, 0), lane = tid & 31;
-#ifdef BASP_PHASE_TIMING
-    long long bacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-#endif
 
     if (tid == 0) {
         mbar_init(&bars->kv_full, 1); mbar_init(&bars->kv_empty, 1);
@@ -75,11 +72,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_d64_kernel(const __gr
                     const int buf = it_g & 1;                                   // S^T buffer of the step
                     const uint32_t stage = it_g % kQS, sph = (it_g / kQS) & 1;  // its Q / dO stage (row statistics with it)
                     const uint32_t st_col = tmem + kColST + 128 * buf + 32 * g + lane_addr;
-                    BPH_T(t0);
                     BWD_WAIT(&bars->stats_full[stage], sph, 10, m);             // LSE and Delta of the query tile
                     BWD_WAIT(&bars->s_full_b[buf], (it_g >> 1) & 1, 11, m);
                     tc_fence_after();
-                    BPH_T(t1);
                     uint32_t st[32], dp[32];
                     tmem_ld_x32(st_col, st);
                     tmem_wait_ld();
@@ -126,10 +121,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_d64_kernel(const __gr
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars->p_ready);          // product (3) of this step may start
                     // dS^T = P^T (dP^T scale - Delta scale): dP^T arrives after dQ of the step before has left TMEM
-                    BPH_T(t2);
                     BWD_WAIT(&bars->dp_full, it_g & 1, 12, m);
                     tc_fence_after();
-                    BPH_T(t3);
                     tmem_ld_x32(tmem + kColDP + 32 * g + lane_addr, dp);
                     tmem_wait_ld();
 #pragma unroll
@@ -157,8 +150,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_d64_kernel(const __gr
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars->pds_ready);
-                    BPH_T(t4);
-                    BPH_ADD(0, t0, t1); BPH_ADD(1, t1, t2); BPH_ADD(2, t2, t3); BPH_ADD(3, t3, t4); BPH_ADD(6, t0, t0 + 1);
                 }
             }
             // ---- item done: dK_n (quarters 0, 1) / dV_n (quarters 2, 3) to global as bf16, 32 columns per quarter
@@ -200,10 +191,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_d64_kernel(const __gr
             for (int hq = 0; hq < p.q_per_kv; ++hq) {
                 const int h = item.hkv * p.q_per_kv + hq;
                 for (int m = item.m0; m < item.n_qt; ++m, ++it_g) {
-                    BPH_T(v0);
                     BWD_WAIT(&bars->dq_full, it_g & 1, 14, m);
                     tc_fence_after();
-                    BPH_T(v1);
                     uint32_t v[64];
                     tmem_ld_x32(tmem + kColDP + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
                     tmem_ld_x32(tmem + kColDP + 32 + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
@@ -232,8 +221,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_d64_kernel(const __gr
                         tma_store_wait_read<0>();
                     }
                     __syncwarp();
-                    BPH_T(v2);
-                    BPH_ADD(0, v0, v1); BPH_ADD(1, v1, v2); BPH_ADD(6, v0, v0 + 1);
                 }
             }
         }
@@ -357,10 +344,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_d64_kernel(const __gr
             for (uint32_t j = 0; j < steps; ++j) {
                 const uint32_t it = it_g + j, stage = it % kQS;
                 const uint32_t q16 = aQ + stage * (kTileBytes >> 4);
-                BPH_T(u0);
                 BWD_WAIT(&bars->pds_ready, it & 1, 33, (int)j);
                 tc_fence_after();
-                BPH_T(u1);
                 if (lane == 0) {
                     const uint32_t acc0 = j == 0 ? 0u : 1u;
                     // (5) dQ_m = dS K : A = the dS^T buffer read MN-major (query rows), B = K MN-major
@@ -378,13 +363,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_d64_kernel(const __gr
                     }
                     tc_commit(&bars->qdo_mma_done[stage]);        // (3), issued a step ago, and (4) are done: the stage may be loaded again
                 }
-                BPH_T(u2);
                 ok = true;
                 if (j + 1 < steps) ok = issue_dp(it + 1) && issue_dv(it + 1, false);
-                BPH_T(u3);
                 if (ok && j + 2 < steps) ok = issue_s(it + 2);
-                BPH_T(u4);
-                BPH_ADD(0, u0, u1); BPH_ADD(1, u1, u2); BPH_ADD(2, u2, u3); BPH_ADD(3, u3, u4); BPH_ADD(6, u0, u0 + 1);
                 if (!ok) { bars->abort_flag = 1; bwd_report(p.status, 3, 35, (int)j); goto bwd_done; }
             }
             it_g += steps;
@@ -397,12 +378,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_d64_kernel(const __gr
     }
 
 bwd_done:
-#ifdef BASP_PHASE_TIMING
-    if (blockIdx.x == 5 && (threadIdx.x & 31) == 0 && (warp == 0 || warp == kBwdMmaWarp || warp == kBwdDrainWarp0)) {
-        const int base_ = warp == 0 ? 0 : (warp == kBwdMmaWarp ? 8 : 16);
-        for (int i_ = 0; i_ < 8; ++i_) g_bwd_phase[base_ + i_] += bacc[i_];
-    }
-#endif
     tc_fence_before();
     __syncthreads();
     if (bars->abort_flag) {

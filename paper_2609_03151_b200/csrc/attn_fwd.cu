@@ -23,14 +23,6 @@ int *basp_status_device_ptr();
 #define BASP_BAND_TARGET 32   // CTAs that share one KV stream at a time (query blocks per band x query heads per KV head)
 #endif
 
-#ifdef BASP_PHASE_TIMING
-extern "C" int basp_debug_phases(long long *out, int reset) {
-    if (out && cudaMemcpyFromSymbol(out, g_phase_cycles, sizeof(long long) * 64) != cudaSuccess) return -1;
-    if (reset) { long long z[64] = {0}; if (cudaMemcpyToSymbol(g_phase_cycles, z, sizeof(z)) != cudaSuccess) return -1; }
-    return 0;
-}
-#endif
-
 namespace {
 
 template <int R>

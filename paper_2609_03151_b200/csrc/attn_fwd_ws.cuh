@@ -32,10 +32,6 @@ namespace {
 constexpr int kWsThreads = 512;
 constexpr int kStages = 4;            // K/V ring slots (one 128 x D tile each)
 constexpr float kRescaleThreshold = 8.f;
-#ifndef BASP_POLY_PAIRS
-#define BASP_POLY_PAIRS 0
-#endif
-constexpr int kPolyPairsOf8 = BASP_POLY_PAIRS;   // of every 8 score pairs, how many take the polynomial exp2
 
 struct WsItem {
     int r, bl, h, hkv, qb;
@@ -87,28 +83,11 @@ struct WsShared {
     int abort_flag;
 };
 
-#ifdef BASP_PHASE_TIMING
-__device__ long long g_phase_cycles[64];
-#define PHASE_T(var) const long long var = clock64()
-#define PHASE_ADD(slot, a, b) do { if (blockIdx.x == 0 && (threadIdx.x & 127) == 0) g_phase_cycles[slot] += (b) - (a); } while (0)
-#define PHASE_ADD1(slot, a, b) do { ph_acc[(slot) - 16] += (b) - (a); } while (0)
-#define PHASE_DECL long long ph_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}
-#define PHASE_FLUSH do { if (blockIdx.x == 0 && lane == 0) for (int i_ = 0; i_ < 8; ++i_) g_phase_cycles[16 + i_] = ph_acc[i_]; } while (0)
-#else
-#define PHASE_T(var)
-#define PHASE_ADD(slot, a, b)
-#define PHASE_ADD1(slot, a, b)
-#define PHASE_DECL
-#define PHASE_FLUSH
-#endif
-
-#ifndef BASP_SLEEP_NS
-#define BASP_SLEEP_NS 32    // back-off of the correction and producer warps while they wait
-#endif
+constexpr uint32_t kSleepNs = 32;     // back-off of the correction and producer warps while they wait
 
 #define WS_WAIT(bar, parity, role, detail)                                     \
     do {                                                                        \
-        if (!mbar_wait((bar), (parity), &sh.abort_flag, ((role) >= 20 && (role) < 40) ? BASP_SLEEP_NS : 0)) { \
+        if (!mbar_wait((bar), (parity), &sh.abort_flag, ((role) >= 20 && (role) < 40) ? kSleepNs : 0)) { \
             sh.abort_flag = 1;                                                  \
             report(p.status, 1, (role), (detail));                              \
             goto ws_done;                                                       \
@@ -172,10 +151,8 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
             if (n_t == 0) continue;
             float m_ref = -INFINITY, l_run = 0.f;
             for (int j = 0; j < n_t; ++j, ++it_cnt) {
-                PHASE_T(c0);
                 WS_WAIT(&sh.s_full[t], it_cnt & 1, 10 + t, j);
                 tc_fence_after();
-                PHASE_T(c1);
                 uint32_t s[kTile];
                 tmem_ld_x32(S_a + 0, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
                 tmem_ld_x32(S_a + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
@@ -185,7 +162,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.s_free);       // the scores are in registers: the other tile's Q.K^T may overwrite S
-                PHASE_T(c2);
                 // Key column i of this tile is visible iff i <= lim: the causal diagonal (i <= row) and, in a
                 // ragged last tile, the end of the sequence (i < S - 128 j; what lies beyond belongs to the next
                 // sequence of the shard or is TMA zero fill).
@@ -219,7 +195,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.alpha_full[t][it_cnt & 1]);
                 m_ref = m_new;
-                PHASE_T(c3);
                 const uint64_t sc2 = pack_f2(p.scale_log2, p.scale_log2), nm2 = pack_f2(-m_new, -m_new);
                 uint64_t rs2[2] = {0ull, 0ull};
                 auto exp_row = [&](auto diag_tag) {
@@ -227,15 +202,9 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
 #pragma unroll
                     for (int i = 0; i < kTile; i += 2) {
                         const uint64_t x2 = fma2(pack_f2(__uint_as_float(s[i]), __uint_as_float(s[i + 1])), sc2, nm2);
-                        float e0, e1;
-                        if (((i >> 1) & 7) < kPolyPairsOf8) {
-                            exp2_poly_pair(x2, e0, e1);
-                        } else {
-                            float x0, x1;
-                            unpack_f2(x2, x0, x1);
-                            e0 = exp2_approx(x0);
-                            e1 = exp2_approx(x1);
-                        }
+                        float x0, x1;
+                        unpack_f2(x2, x0, x1);
+                        float e0 = exp2_approx(x0), e1 = exp2_approx(x1);
                         if (kDiag) {                  // masked keys contribute exactly nothing
                             if (i > lim) e0 = 0.f;
                             if (i + 1 > lim) e1 = 0.f;
@@ -250,7 +219,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 float ra, rb;
                 unpack_f2(add2(rs2[0], rs2[1]), ra, rb);
                 l_run = l_run * alpha + (ra + rb);
-                PHASE_T(c4);
                 // The previous P_t V (of this item or, at j = 0, the last one of the item before) is issued by a warp
                 // of its own: make sure it has read P_t before this step's P_t replaces it.  Waiting at every step
                 // also means that no phase of the barrier is ever skipped.
@@ -261,9 +229,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.p_full[t]);
-                PHASE_T(c5);
-                PHASE_ADD(8 * t + 0, c0, c1); PHASE_ADD(8 * t + 1, c1, c2); PHASE_ADD(8 * t + 2, c2, c3);
-                PHASE_ADD(8 * t + 3, c3, c4); PHASE_ADD(8 * t + 4, c4, c5); PHASE_ADD(8 * t + 5, c0, c0 + 1);
             }
             sh.l[ep_cnt & 1][t][row] = l_run;
             __syncwarp();
@@ -388,23 +353,17 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
             // Descriptors differ only in the 14-bit start-address field, so a step along K is an add.
             const uint64_t desc_k = make_smem_desc_sw128(0, 16, 1024);        // K-major operands (Q, K)
             const uint32_t q_addr16 = smem_u32(sQ) >> 4, kv_addr16 = smem_u32(sKV) >> 4;
-            PHASE_DECL;
             for (int round = 0; ws_get_item(p, round, item); ++round, ++item_n) {
                 WS_WAIT(&sh.q_full, item_n & 1, 40, round);
                 for (int j = 0; j < item.n_max; ++j) {
                     const uint32_t idx = kv_base + 2 * j, slot = idx % kStages;
-                    PHASE_T(k0);
                     WS_WAIT(&sh.kv_full[slot], (idx / kStages) & 1, 41, j);
-                    PHASE_T(k1);
-                    PHASE_ADD1(21, k0, k1);
                     tc_fence_after();
 #pragma unroll
                     for (int t = 0; t < 2; ++t) {
                         if (j >= item.n[t]) continue;
                         // score tile number q may only follow the hand-over of q - 1 to its softmax warps
-                        PHASE_T(q0);
                         if (qk_cnt > 0) { WS_WAIT(&sh.s_free, (qk_cnt - 1) & 1, 48, j); tc_fence_after(); }
-                        PHASE_T(q1);
                         ++qk_cnt;
                         const uint64_t a = desc_k | (uint64_t)(q_addr16 + t * (kTileBytes >> 4));
                         const uint64_t b = desc_k | (uint64_t)(kv_addr16 + slot * (kTileBytes >> 4));
@@ -418,8 +377,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                             }
                             tc_commit(&sh.s_full[t]);
                         }
-                        PHASE_T(q2);
-                        PHASE_ADD1(16, q0, q1); PHASE_ADD1(22, q1, q2); PHASE_ADD1(23, q0, q0 + 1);
                     }
                     if (lane == 0) {
                         tc_commit(&sh.kv_empty[slot]);                            // K_j has no reader left
@@ -428,7 +385,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) attn_fwd_ws_kernel(const __grid
                 }
                 kv_base += 2 * item.n_max;
             }
-            PHASE_FLUSH;
         } else if (warp == 14) {
             // =========================================================== MMA issuer 2: O_t += P_t V_j (lane 0 issues)
             const uint32_t idesc_pv = make_idesc_bf16(kTile, D, false, true);

@@ -240,26 +240,6 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
-// 2^x for a pair without the special-function unit: round-to-nearest split x = n + f with
-// f in [-0.5, 0.5] (magic-number rounding), cubic for 2^f (max relative error 7.5e-5, far below
-// the bf16 rounding the result receives), n added into the exponent field.  x is clamped at -126.
-__device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float &e0, float &e1) {
-    float x0, x1;
-    unpack_f2(x2, x0, x1);
-    x2 = pack_f2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
-    const uint64_t magic = pack_f2(12582912.f, 12582912.f);
-    const uint64_t xr = add2(x2, magic);
-    const uint64_t nf = add2(xr, pack_f2(-12582912.f, -12582912.f));
-    const uint64_t f = fma2(nf, pack_f2(-1.f, -1.f), x2);
-    uint64_t pl = fma2(f, pack_f2(0.0551716610789299f, 0.0551716610789299f), pack_f2(0.2426111251115799f, 0.2426111251115799f));
-    pl = fma2(pl, f, pack_f2(0.6932609677314758f, 0.6932609677314758f));
-    pl = fma2(pl, f, pack_f2(0.9999280571937561f, 0.9999280571937561f));
-    float p0, p1, r0, r1;
-    unpack_f2(pl, p0, p1);
-    unpack_f2(xr, r0, r1);
-    e0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(r0) << 23));
-    e1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(r1) << 23));
-}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));

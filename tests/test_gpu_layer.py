@@ -111,10 +111,26 @@ def test_host_buffer_entry_full_size_sampled_rows(basp, name):
     assert_attn_close(got, ref, f"{name} host entry")
 
 
+def sampled_rows(S, T, B, Hq, seed=0):
+    """Rows checked per (sequence, query head) at full size: rows 0..255 (both sides of the first tile boundaries
+    included), both sides of every shard boundary l*T, the last 256 rows and 64 seeded random rows."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for b in range(B):
+        for h in range(Hq):
+            pos = set(range(min(256, S))) | set(range(max(0, S - 256), S))
+            for edge in range(T, S, T):
+                pos |= {edge - 1, edge}
+            pos |= {int(x) for x in rng.integers(0, S, 64)}
+            out += [(b, h, i) for i in sorted(pos)]
+    return np.array(out, dtype=np.int32)
+
+
 @pytest.mark.parametrize("name", ["llama3_8b_32k", "sweep_b1", "sweep_b4", "sweep_b8", "qwen25_7b_64k"])
 def test_full_size_sampled_rows(basp, name):
-    """BASELINE configs 2, 3 (b = 1, 4, 8; b = 2 is config 2) and 4 at full size, the launches the benchmark times:
-    sampled output rows (first rows, shard and tile boundaries, last rows, random rows) against oracle rows."""
+    """The Llama-3-8B shape at 32K with two groups of four, the same shape with 65536 tokens over 1, 4 and 8 sequences,
+    and the Qwen2.5-7B shape at 64K, at full size through the launches the benchmark times: per (sequence, query head)
+    rows 0..255, both sides of every shard boundary, the last 256 rows and 64 random rows against oracle rows."""
     w = synth.WORKLOADS[name]
     q, k, v = synth.make_qkv(w, seed=0)
     pl = make_plan(basp, w)
@@ -124,12 +140,7 @@ def test_full_size_sampled_rows(basp, name):
         return [x[r // K: r // K + 1, (r % K) * T:(r % K + 1) * T].contiguous().cuda() for r in range(w.N)]
 
     dq, dk, dv = shards(q), shards(k), shards(v)
-    rng = np.random.default_rng(0)
-    cand = sorted({i for i in (0, 1, 127, 128, 255, 256, T - 1, T, T + 1, 2 * T - 1, 2 * T, w.S - 129, w.S - 128, w.S - 1)
-                   if i < w.S})
-    rows = [(b, h, i) for b in range(w.B) for h in (0, 5, w.Hq - 1) for i in cand]
-    rows += [(int(rng.integers(w.B)), int(rng.integers(w.Hq)), int(rng.integers(w.S))) for _ in range(40)]
-    rows = np.array(rows, dtype=np.int32)
+    rows = sampled_rows(w.S, T, w.B, w.Hq)
     ref, _ = oracle.attn_fwd_rows(synth.bits(q), synth.bits(k), synth.bits(v), rows)
     ws = torch.empty(basp.basp_workspace_bytes(pl), dtype=torch.uint8, device="cuda")
     for fused in (False, True):
@@ -140,7 +151,9 @@ def test_full_size_sampled_rows(basp, name):
         else:
             basp.basp_layer_fwd(pl, dq, dk, dv, do, ws)
         basp.basp_get_status()
-        got = np.stack([do[b * K + i // T][0, i % T, h].float().cpu().numpy().astype(np.float64) for b, h, i in rows])
+        flat = torch.stack(do).reshape(w.B, w.S, w.Hq, w.D)          # the shards in rank order are the global tensor
+        ix = torch.from_numpy(rows.astype(np.int64)).cuda()
+        got = flat[ix[:, 0], ix[:, 2], ix[:, 1]].float().cpu().numpy().astype(np.float64)
         assert_attn_close(got, ref, f"{name} fused={fused}")
 
 
