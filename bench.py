@@ -3,13 +3,21 @@
 
 One step = one pass of the layer over one synthetic micro-batch held as N virtual ranks on one
 GPU: all-to-all reshard of Q, K, V (sequence- to head-sharded), causal attention over every rank's
-head slice, reverse reshard of O.  Prints ONE JSON line (rank 0).
+head slice, reverse reshard of O (and, for a training workload, the backward: exchange of dO, attention
+backward, reverse exchanges of dQ, dK, dV).  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
+The headline is the largest forward-only shape (Qwen2.5-7B heads, 64K tokens, two groups of four).  With one GPU
+the line also carries `configs`: every benchmark shape (tiny; Llama-3-8B at 32K; the 65536-token sweep over
+b = 1, 2, 4, 8; Qwen2.5-7B at 64K; the 128K-token training step) timed in the same run, each with its kernel rates,
+its fused form, its end-to-end number and the clocks sampled during that leg; and `span`: the layer of one group of
+eight ranks through the entry points that serve a group spread over GPUs (on one GPU: every rank local).
+
 With --gpus N > 1 (launched by torchrun, one process per GPU) every GPU runs its own micro-batch
 of the same shape (weak scaling; BASP groups and micro-batches are independent, so the data path
-has no collective); times are the maximum over ranks.
+has no collective); times are the maximum over ranks.  The `span` leg then spreads ONE micro-batch's group of eight
+ranks over the N GPUs (peer loads and stores over NVLink, no collective library on the data path).
 """
 from __future__ import annotations
 
@@ -32,13 +40,30 @@ from paper_2609_03151_b200 import synth  # noqa: E402
 
 METRIC = "attention-layer tokens/sec"
 UNIT = "tokens/s"
-DEFAULT_WORKLOAD = "llama3_8b_32k"          # BASELINE config 2: N=8, b=2, S=32768, 32/8 heads, D=128
+DEFAULT_WORKLOAD = "qwen25_7b_64k"          # N=8, b=2 (groups of 4), S=65536, 28/4 heads, D=128: the largest forward shape
+ALL_SHAPES = ["tiny", "llama3_8b_32k", "sweep_b1", "sweep_b2", "sweep_b4", "sweep_b8", "qwen25_7b_64k",
+              "llama3_8b_128k_train"]
+SPAN_WORKLOAD = "sweep_b1"                  # one group of eight ranks: the shape whose exchange crosses GPUs
 
-# DRAM bytes (read + write) of one attention launch from an ncu capture, per workload; None = not captured.
-NCU_TRAFFIC_BYTES = {
-    # profiles/attn_fwd_ws_traffic_llama3_8b_32k.md: dram__bytes_read.sum + dram__bytes_write.sum of one launch
-    "llama3_8b_32k": 3033940992 + 539852800,
-}
+
+def ncu_traffic(workload: str, kernel: str):
+    """DRAM bytes (read + write) of one launch of `kernel` on `workload` from the profiler capture that the tracked
+    table names, or None where no capture exists."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    try:
+        entry = json.load(open(path))[workload][kernel]
+        return int(entry["dram_bytes_read"]) + int(entry["dram_bytes_write"])
+    except (OSError, KeyError, ValueError):
+        return None
+
+
+def config_dict(w: synth.Workload) -> dict:
+    """The workload description both arms print."""
+    path = ("forward (s2h, attn_fwd, h2s) + backward (s2h dO, attn_bwd, h2s dQ/dK/dV)" if w.train
+            else "reshard_qkv_s2h -> attn_fwd -> reshard_h2s (3 launches/step)")
+    return {"workload": w.name, "N": w.N, "b": w.B, "group_size": w.K, "S": w.S, "Hq": w.Hq, "Hkv": w.Hkv, "D": w.D,
+            "causal": True, "path": path, "l2": "inputs larger than L2 (no flush needed)" if w.name != "tiny" else
+            "tiny shape: L2-resident, launch-bound (no roofline claimed)", "per_gpu_tokens": w.tokens}
 
 
 def measured_peaks():
@@ -151,12 +176,268 @@ def run_reference(args, w: synth.Workload):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.tokens / value,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "N": w.N, "b": w.B, "S": w.S, "Hq": w.Hq, "Hkv": w.Hkv, "D": w.D,
-                       "note": "fp64 CPU oracle on a bounded sample per step, extrapolated"},
+            "config": config_dict(w), "note": "fp64 CPU oracle on a bounded sample per step, extrapolated",
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
+
+
+
+
+# ------------------------------------------------------------------------------------------
+class Shape:
+    """Device buffers of one workload on one GPU: sequence-sharded inputs drawn N(0,1) -> bf16 per shard from a seeded
+    device generator (timing only; the parity tests use the CPU generator on global coordinates), head-sharded
+    intermediates, and for a training workload the gradients and the backward workspace."""
+
+    def __init__(self, basp, w: synth.Workload, dev, seed: int):
+        self.w, self.basp = w, basp
+        self.plan = plan = basp.basp_plan_create(w.N, w.B, w.S, w.Hq, w.Hkv, w.D, num_groups=w.G)
+        N, T, Bl = w.N, plan.T, plan.Bl
+        gen = torch.Generator(device=dev).manual_seed(seed)
+        self.randn = lambda shape: torch.randn(shape, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        empty = lambda shape: torch.empty(shape, dtype=torch.bfloat16, device=dev)
+        self.q_seq = [self.randn((Bl, T, w.Hq, w.D)) for _ in range(N)]
+        self.k_seq = [self.randn((Bl, T, w.Hkv, w.D)) for _ in range(N)]
+        self.v_seq = [self.randn((Bl, T, w.Hkv, w.D)) for _ in range(N)]
+        self.o_seq = [torch.empty_like(t) for t in self.q_seq]
+        self.q_head = [empty((Bl, w.S, plan.Hq_l, w.D)) for _ in range(N)]
+        self.k_head = [empty((Bl, w.S, plan.Hkv_l, w.D)) for _ in range(N)]
+        self.v_head = [empty((Bl, w.S, plan.Hkv_l, w.D)) for _ in range(N)]
+        self.o_head = [torch.empty_like(t) for t in self.q_head]
+        self.lse = None
+        if w.train:
+            self.do_seq = [self.randn((Bl, T, w.Hq, w.D)) for _ in range(N)]
+            self.do_head = [torch.empty_like(t) for t in self.q_head]
+            self.dq_head = [torch.empty_like(t) for t in self.q_head]
+            self.dk_head = [torch.empty_like(t) for t in self.k_head]
+            self.dv_head = [torch.empty_like(t) for t in self.k_head]
+            self.dq_seq = [torch.empty_like(t) for t in self.q_seq]
+            self.dk_seq = [torch.empty_like(t) for t in self.k_seq]
+            self.dv_seq = [torch.empty_like(t) for t in self.k_seq]
+            self.lse = [torch.empty((Bl, plan.Hq_l, w.S), dtype=torch.float32, device=dev) for _ in range(N)]
+            self.bwd_ws = torch.empty(basp.basp_attn_bwd_workspace_bytes(plan), dtype=torch.uint8, device=dev)
+        self.n_events = 7 if w.train else 4
+
+    def step(self, events=None):
+        """a2 -> a3 -> a4 (what basp_layer_fwd launches) and, for a training workload, a7 -> a6 -> a7 (what
+        basp_layer_bwd launches), with optional events between the launches."""
+        b, p, w = self.basp, self.plan, self.w
+
+        def mark(i):
+            if events:
+                events[i].record()
+        mark(0)
+        b.basp_reshard_qkv_s2h(p, self.q_seq, self.k_seq, self.v_seq, self.q_head, self.k_head, self.v_head)
+        mark(1)
+        b.basp_attn_fwd(p, self.q_head, self.k_head, self.v_head, self.o_head, self.lse)
+        mark(2)
+        b.basp_reshard_h2s(p, w.Hq, self.o_head, self.o_seq)
+        mark(3)
+        if w.train:
+            b.basp_reshard_s2h(p, w.Hq, self.do_seq, self.do_head)
+            mark(4)
+            b.basp_attn_bwd(p, self.q_head, self.k_head, self.v_head, self.o_head, self.do_head, self.lse, self.dq_head,
+                            self.dk_head, self.dv_head, self.bwd_ws)
+            mark(5)
+            b.basp_reshard_grads_h2s(p, self.dq_head, self.dk_head, self.dv_head, self.dq_seq, self.dk_seq, self.dv_seq)
+            mark(6)
+
+
+def time_steps(shape: Shape, steps: int, warmup: int, rank: int, local_rank: int):
+    """W untimed steps, then exactly `steps` timed ones between barriers and device synchronisations, CUDA events on the
+    launching stream around every launch, the clocks sampled meanwhile.  Returns a dict of per-launch means (ms)."""
+    basp = shape.basp
+    basp.basp_clear_status()
+    for _ in range(warmup):
+        shape.step()
+    torch.cuda.synchronize()
+    basp.basp_get_status()
+    n_ev = shape.n_events
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(n_ev)] for _ in range(steps)]
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    launches0 = basp.basp_launch_count()
+    pdist.barrier()
+    torch.cuda.synchronize()
+    for i in range(steps):
+        shape.step(ev[i])
+    torch.cuda.synchronize()
+    pdist.barrier()
+    launches = basp.basp_launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    basp.basp_get_status()
+    mean = lambda i: statistics.mean(e[i].elapsed_time(e[i + 1]) for e in ev)
+    per_step = [e[0].elapsed_time(e[n_ev - 1]) for e in ev]
+    out = {"total_ms": ev[0][0].elapsed_time(ev[-1][n_ev - 1]), "per_step": per_step, "launches": launches, "clocks": clocks,
+           "ms_s2h": mean(0), "ms_attn": mean(1), "ms_h2s": mean(2)}
+    if shape.w.train:
+        out.update(ms_s2h_do=mean(3), ms_attn_bwd=mean(4), ms_h2s_grads=mean(5))
+    return out
+
+
+def time_fused(shape: Shape, steps: int, warmup: int) -> float:
+    """basp_layer_fwd_fused (one kernel straight from / to the sequence-sharded shards): ms per call."""
+    b = shape.basp
+    for _ in range(max(1, warmup // 2)):
+        b.basp_layer_fwd_fused(shape.plan, shape.q_seq, shape.k_seq, shape.v_seq, shape.o_seq)
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    f0.record()
+    for _ in range(steps):
+        b.basp_layer_fwd_fused(shape.plan, shape.q_seq, shape.k_seq, shape.v_seq, shape.o_seq)
+    f1.record()
+    torch.cuda.synchronize()
+    b.basp_get_status()
+    return f0.elapsed_time(f1) / steps
+
+
+def time_e2e_host(shape: Shape, steps: int, dev):
+    """End to end through the C ABI with HOST buffers: basp_layer_fwd_host copies the pinned Q, K, V shards to the device,
+    runs the fused kernel per arrived piece and copies O back, all inside the timed region (wall clock around the
+    synchronous call).  Returns (ms per call, H2D bytes, D2H bytes)."""
+    b, plan = shape.basp, shape.plan
+    hq = [t.cpu().pin_memory() for t in shape.q_seq]
+    hk = [t.cpu().pin_memory() for t in shape.k_seq]
+    hv = [t.cpu().pin_memory() for t in shape.v_seq]
+    ho = [torch.empty_like(t).pin_memory() for t in hq]
+    arena = torch.empty(b.basp_host_arena_bytes(plan), dtype=torch.uint8, device=dev)
+    b.basp_layer_fwd_host(plan, hq, hk, hv, ho, arena)
+    pdist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        b.basp_layer_fwd_host(plan, hq, hk, hv, ho, arena)       # synchronises the stream itself
+    torch.cuda.synchronize()
+    ms = (time.perf_counter() - t0) * 1e3 / steps
+    return ms, sum(t.numel() * 2 for t in hq + hk + hv), sum(t.numel() * 2 for t in ho)
+
+
+def time_e2e_train(shape: Shape, steps: int, dev):
+    """The training step through the layer entry points of the C ABI (basp_layer_fwd, then basp_layer_bwd on the
+    head-sharded activations the forward left in its workspace), wall clock around the calls and a device
+    synchronisation.  The activations and the loss gradient of a training step are produced and consumed on the
+    device by the layers around this one, so the step has no host boundary: zero bytes cross the bus."""
+    b, plan, w = shape.basp, shape.plan, shape.w
+    ws = torch.empty(b.basp_workspace_bytes(plan), dtype=torch.uint8, device=dev)
+    ws2 = torch.empty(b.basp_layer_bwd_workspace_bytes(plan), dtype=torch.uint8, device=dev)
+
+    def one():
+        b.basp_layer_fwd(plan, shape.q_seq, shape.k_seq, shape.v_seq, shape.o_seq, ws, shape.lse)
+        qh, kh, vh, oh = (b.as_shards(a) for a in b.basp_layer_workspace_shards(plan, ws))
+        b.basp_layer_bwd(plan, qh, kh, vh, oh, shape.lse, shape.do_seq, shape.dq_seq, shape.dk_seq, shape.dv_seq, ws2)
+    one()
+    torch.cuda.synchronize()
+    pdist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one()
+    torch.cuda.synchronize()
+    ms = (time.perf_counter() - t0) * 1e3 / steps
+    b.basp_get_status()
+    return ms
+
+
+def rates(w: synth.Workload, t: dict, peaks: dict) -> dict:
+    """Kernel rates of one timed shape: attention TFLOP/s against the measured sustained and burst cuBLAS bf16 rates and
+    the nominal 2250, both exchanges in GB/s against the measured copy bandwidth and the nominal 8 TB/s."""
+    def tensor(flops, ms):
+        tf = flops / (ms * 1e-3) / 1e12
+        return {"ms": ms, "tflops": tf, "frac_of_sustained": tf / peaks["bf16_sustained"],
+                "frac_of_burst": tf / peaks["bf16_burst"], "frac_of_nominal_2250": tf / 2250.0}
+
+    def hbm(nbytes, ms):
+        g = nbytes / (ms * 1e-3) / 1e9
+        return {"ms": ms, "gbs": g, "frac_of_measured_copy": g / peaks["hbm_gbs"], "frac_of_nominal_8000": g / 8000.0,
+                "bytes": nbytes}
+    out = {"attn_fwd": tensor(w.attn_flops_fwd(), t["ms_attn"]),
+           "reshard_qkv_s2h": hbm(w.reshard_bytes_s2h(), t["ms_s2h"]),
+           "reshard_h2s": hbm(w.reshard_bytes_h2s(), t["ms_h2s"])}
+    if w.train:
+        out["attn_bwd"] = tensor(w.attn_flops_bwd(), t["ms_attn_bwd"])
+        out["attn_bwd"]["launches"] = "memset + Delta + main kernel + dQ conversion"
+        out["reshard_s2h_do"] = hbm(w.reshard_bytes_h2s(), t["ms_s2h_do"])
+        out["reshard_grads_h2s"] = hbm(w.reshard_bytes_s2h(), t["ms_h2s_grads"])
+    return out
+
+
+def measure_shape(basp, w: synth.Workload, dev, rank: int, local_rank: int, steps: int, warmup: int, peaks: dict,
+                  e2e_steps: int = 3) -> dict:
+    """One entry of `configs`: the three-launch step (plus the backward for a training shape), the fused form, the
+    end-to-end number, rates and clocks of one shape."""
+    shape = Shape(basp, w, dev, seed=1000 + rank)
+    t = time_steps(shape, steps, warmup, rank, local_rank)
+    ms = t["total_ms"] / steps
+    entry = {"config": config_dict(w), "steps": steps, "warmup": warmup, "ms_per_step": ms,
+             "tokens_per_s": w.tokens / (ms * 1e-3), "kernels": rates(w, t, peaks), "clocks": t["clocks"],
+             "gpu_launches": t["launches"]}
+    if w.train:
+        e_ms = time_e2e_train(shape, min(steps, e2e_steps), dev)
+        entry["e2e"] = {"ms_per_step": e_ms, "value": w.tokens / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 0,
+                        "d2h_bytes_per_step": 0,
+                        "call": "basp_layer_fwd + basp_layer_bwd from device buffers (a training step has no host boundary)"}
+    else:
+        f_ms = time_fused(shape, steps, warmup)
+        entry["fused"] = {"ms_per_step": f_ms, "tokens_per_s": w.tokens / (f_ms * 1e-3),
+                          "tflops": w.attn_flops_fwd() / (f_ms * 1e-3) / 1e12,
+                          "ms_minus_attention_launch": f_ms - t["ms_attn"]}
+        del shape.q_head, shape.k_head, shape.v_head, shape.o_head
+        e_ms, h2d, d2h = time_e2e_host(shape, min(steps, e2e_steps), dev)
+        entry["e2e"] = {"ms_per_step": e_ms, "value": w.tokens / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": d2h, "call": "basp_layer_fwd_host (pinned host shards)"}
+    del shape
+    torch.cuda.empty_cache()
+    return entry
+
+
+def measure_span(basp, dev, rank: int, world: int, steps: int, warmup: int) -> dict:
+    """One micro-batch whose single group of eight ranks is spread over the GPUs of the run (on one GPU: all eight
+    local): the fused form (Q/K/V tiles fetched from wherever the group's sequence shards live, O tiles stored into
+    the owner's shard) and the three-step form (push exchange, attention, pull exchange), both through the `*_ranks`
+    entry points over a symmetric shard table, host barriers between the steps.  Peer loads and stores only."""
+    w = synth.WORKLOADS[SPAN_WORKLOAD]
+    if w.N % world != 0:
+        return {"skipped": f"{w.N} ranks do not divide over {world} GPUs"}
+    plan = basp.basp_plan_create(w.N, w.B, w.S, w.Hq, w.Hkv, w.D)
+    T, S = plan.T, w.S
+    qb, kb = T * w.Hq * w.D * 2, T * w.Hkv * w.D * 2
+    qhb, khb = S * plan.Hq_l * w.D * 2, S * plan.Hkv_l * w.D * 2
+    sh = pdist.SymmetricShards(w.N, {"q": qb, "k": kb, "v": kb, "o": qb, "qh": qhb, "kh": khb, "vh": khb, "oh": qhb})
+    gen = torch.Generator(device=dev).manual_seed(2000 + rank)
+    for r in sh.local:
+        for name in ("q", "k", "v"):
+            t = sh.local_shard(name, r).view(torch.bfloat16)
+            t.copy_(torch.randn(t.shape, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16))
+    out = {"workload": w.name, "group_size": plan.K, "gpus": world, "ranks_per_gpu": len(sh.local),
+           "remote_fraction_of_exchange_bytes": sh.remote_fraction(plan.K), "tokens": w.tokens}
+    basp.basp_clear_status()
+    for name, fn in (("fused", pdist.layer_fwd_fused_multi_gpu), ("three_step", pdist.layer_fwd_three_step_multi_gpu)):
+        for _ in range(max(1, warmup // 2)):
+            fn(plan, sh)
+        torch.cuda.synchronize()
+        pdist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            fn(plan, sh)
+        torch.cuda.synchronize()
+        ms = pdist.max_over_ranks((time.perf_counter() - t0) * 1e3 / steps)
+        out[name] = {"ms_per_step": ms, "tokens_per_s": w.tokens / (ms * 1e-3)}
+        if name == "fused":
+            fused_o = [sh.local_shard("o", r).clone() for r in sh.local]
+    basp.basp_get_status()
+    same = all(torch.equal(a, sh.local_shard("o", r)) for a, r in zip(fused_o, sh.local))
+    out["three_step_equals_fused_bitwise"] = bool(same)
+    if world == 1:      # every rank local: the call must reproduce the single-GPU fused layer bit for bit
+        view = lambda name, r, h: sh.local_shard(name, r).view(torch.bfloat16).view(1, T, h, w.D)
+        q, k, v = ([view(n, r, h) for r in range(w.N)] for n, h in (("q", w.Hq), ("k", w.Hkv), ("v", w.Hkv)))
+        o = [torch.empty_like(t) for t in q]
+        basp.basp_layer_fwd_fused(plan, q, k, v, o)
+        torch.cuda.synchronize()
+        out["equals_single_gpu_fused_bitwise"] = bool(all(torch.equal(a.view(torch.uint8).reshape(-1), b)
+                                                          for a, b in zip(o, fused_o)))
+    del sh
+    torch.cuda.empty_cache()
+    return out
 
 
 # ------------------------------------------------------------------------------------------
@@ -170,281 +451,124 @@ def run_gpu(args, w: synth.Workload):
     dev = torch.device("cuda", local_rank)
     peaks = measured_peaks()
 
-    plan = basp.basp_plan_create(w.N, w.B, w.S, w.Hq, w.Hkv, w.D, num_groups=w.G)
-    N, K, T, Bl = w.N, plan.K, plan.T, plan.Bl
-    gen = torch.Generator(device=dev).manual_seed(1000 + rank)
-
-    def randn(shape):
-        return torch.randn(shape, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
-
-    # sequence-sharded inputs, one allocation per virtual rank (N(0,1) -> bf16, seeded per GPU)
-    q_seq = [randn((Bl, T, w.Hq, w.D)) for _ in range(N)]
-    k_seq = [randn((Bl, T, w.Hkv, w.D)) for _ in range(N)]
-    v_seq = [randn((Bl, T, w.Hkv, w.D)) for _ in range(N)]
-    o_seq = [torch.empty_like(t) for t in q_seq]
-    q_head = [torch.empty((Bl, w.S, plan.Hq_l, w.D), dtype=torch.bfloat16, device=dev) for _ in range(N)]
-    k_head = [torch.empty((Bl, w.S, plan.Hkv_l, w.D), dtype=torch.bfloat16, device=dev) for _ in range(N)]
-    v_head = [torch.empty((Bl, w.S, plan.Hkv_l, w.D), dtype=torch.bfloat16, device=dev) for _ in range(N)]
-    o_head = [torch.empty_like(t) for t in q_head]
-
-    train = w.train
-    if train:
-        do_seq = [randn((Bl, T, w.Hq, w.D)) for _ in range(N)]
-        do_head = [torch.empty_like(t) for t in q_head]
-        dq_head = [torch.empty_like(t) for t in q_head]
-        dk_head = [torch.empty_like(t) for t in k_head]
-        dv_head = [torch.empty_like(t) for t in k_head]
-        dq_seq = [torch.empty_like(t) for t in q_seq]
-        dk_seq = [torch.empty_like(t) for t in k_seq]
-        dv_seq = [torch.empty_like(t) for t in k_seq]
-        lse = [torch.empty((Bl, plan.Hq_l, w.S), dtype=torch.float32, device=dev) for _ in range(N)]
-        bwd_ws = torch.empty(basp.basp_attn_bwd_workspace_bytes(plan), dtype=torch.uint8, device=dev)
-    n_ev = 7 if train else 4
-
-    def step(events=None):
-        """a2 -> a3 -> a4 (what basp_layer_fwd launches) and, for a training workload, a7 -> a6 -> a7
-        (what basp_layer_bwd launches), with optional events between the launches."""
-        def mark(i):
-            if events:
-                events[i].record()
-        mark(0)
-        basp.basp_reshard_qkv_s2h(plan, q_seq, k_seq, v_seq, q_head, k_head, v_head)
-        mark(1)
-        basp.basp_attn_fwd(plan, q_head, k_head, v_head, o_head, lse if train else None)
-        mark(2)
-        basp.basp_reshard_h2s(plan, w.Hq, o_head, o_seq)
-        mark(3)
-        if train:
-            basp.basp_reshard_s2h(plan, w.Hq, do_seq, do_head)
-            mark(4)
-            basp.basp_attn_bwd(plan, q_head, k_head, v_head, o_head, do_head, lse, dq_head, dk_head, dv_head, bwd_ws)
-            mark(5)
-            basp.basp_reshard_grads_h2s(plan, dq_head, dk_head, dv_head, dq_seq, dk_seq, dv_seq)
-            mark(6)
-
-    basp.basp_clear_status()
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
-    basp.basp_get_status()
-
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(n_ev)] for _ in range(args.steps)]
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    launches0 = basp.basp_launch_count()
-    pdist.barrier()
-    torch.cuda.synchronize()
-    for i in range(args.steps):
-        step(ev[i])
-    torch.cuda.synchronize()
-    pdist.barrier()
-    launches = basp.basp_launch_count() - launches0
-    total_ms = ev[0][0].elapsed_time(ev[-1][n_ev - 1])
-    per_step = [e[0].elapsed_time(e[n_ev - 1]) for e in ev]          # each step on its own (the headline is total / steps)
-    ms_s2h = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
-    ms_attn = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
-    ms_h2s = statistics.mean(e[2].elapsed_time(e[3]) for e in ev)
-    ms_bwd = [statistics.mean(e[i].elapsed_time(e[i + 1]) for e in ev) for i in (3, 4, 5)] if train else None
-    basp.basp_get_status()
-
-    proj = None
-    if args.proj:      # the projections on either side of the core (not part of the step): X W_qkv^T and O W_o^T
-        hidden = w.Hq * w.D
-        xs = [randn((Bl * T, hidden)) for _ in range(N)]
-        w_qkv = (torch.randn(((w.Hq + 2 * w.Hkv) * w.D, hidden), generator=gen, device=dev) / hidden ** 0.5).to(torch.bfloat16)
-        w_o = (torch.randn((hidden, w.Hq * w.D), generator=gen, device=dev) / hidden ** 0.5).to(torch.bfloat16)
-        ys = [torch.empty((Bl * T, hidden), dtype=torch.bfloat16, device=dev) for _ in range(N)]
-        pe = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
-        for it in range(args.warmup + args.steps):
-            if it == args.warmup:
-                pe[0].record()
-            basp.basp_qkv_proj(plan, hidden, xs, w_qkv, q_seq, k_seq, v_seq)
-        pe[1].record()
-        for it in range(args.steps):
-            basp.basp_out_proj(plan, hidden, o_seq, w_o, ys)
-        pe[2].record()
-        ms_rope = None
-        if w.D in (64, 128):      # the same projection with rotary position embedding in its epilogue
-            cos, sin = (t.t().contiguous().to(dev) for t in synth.rope_tables(w.S, w.D))      # feature-major
-            re = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-            for it in range(args.warmup + args.steps):
-                if it == args.warmup:
-                    re[0].record()
-                basp.basp_qkv_proj_rope(plan, hidden, xs, w_qkv, cos, sin, q_seq, k_seq, v_seq)
-            re[1].record()
-            torch.cuda.synchronize()
-            ms_rope = re[0].elapsed_time(re[1]) / args.steps
-        torch.cuda.synchronize()
-        basp.basp_get_status()
-        ms_qkv, ms_out = pe[0].elapsed_time(pe[1]) / args.steps, pe[1].elapsed_time(pe[2]) / args.steps
-        f_qkv = 2.0 * N * Bl * T * hidden * (w.Hq + 2 * w.Hkv) * w.D
-        f_out = 2.0 * N * Bl * T * hidden * w.Hq * w.D
-        proj = {"hidden": hidden, "qkv_ms": ms_qkv, "qkv_tflops": f_qkv / ms_qkv / 1e9, "out_ms": ms_out,
-                "out_tflops": f_out / ms_out / 1e9, "qkv_rope_ms": ms_rope,
-                "qkv_rope_tflops": f_qkv / ms_rope / 1e9 if ms_rope else None, "peak_sustained": peaks["bf16_sustained"]}
-        del xs, ys, w_qkv, w_o
-
-    if args.quick:     # kernel timings only (what the ncu recipes in profiles/ run)
-        clocks = sampler.stop() if sampler else None
+    if args.quick:     # kernel timings of one shape only (what the profiler recipes in profiles/ run)
+        shape = Shape(basp, w, dev, seed=1000 + rank)
+        t = time_steps(shape, args.steps, args.warmup, rank, local_rank)
+        proj = time_projections(basp, shape, args, dev) if args.proj else None
         if rank == 0:
-            print(json.dumps({"workload": w.name, "ms_per_step": total_ms / args.steps, "ms_s2h": ms_s2h,
-                              "ms_attn": ms_attn, "ms_h2s": ms_h2s, "gpu_launches": launches,
-                              "attn_tflops": w.attn_flops_fwd() / ms_attn / 1e9, "clocks": clocks,
-                              "bwd_ms_s2h_attn_h2s": ms_bwd, "projections": proj,
-                              "attn_bwd_tflops": (w.attn_flops_bwd() / ms_bwd[1] / 1e9) if train else None}), flush=True)
+            k = rates(w, t, peaks)
+            print(json.dumps({"workload": w.name, "ms_per_step": t["total_ms"] / args.steps, "ms_s2h": t["ms_s2h"],
+                              "ms_attn": t["ms_attn"], "ms_h2s": t["ms_h2s"], "gpu_launches": t["launches"],
+                              "attn_tflops": k["attn_fwd"]["tflops"], "clocks": t["clocks"],
+                              "bwd_ms_s2h_attn_h2s": [t["ms_s2h_do"], t["ms_attn_bwd"], t["ms_h2s_grads"]] if w.train else None,
+                              "projections": proj,
+                              "attn_bwd_tflops": k["attn_bwd"]["tflops"] if w.train else None}), flush=True)
         pdist.finalize()
         return
 
-    if train:
-        return finish_train(args, w, basp, peaks, rank, world, sampler, launches, total_ms, ms_s2h, ms_attn, ms_h2s, ms_bwd, K)
-
-    # fused layer (a5): one kernel straight from / to the sequence-sharded shards
-    for _ in range(max(1, args.warmup // 2)):
-        basp.basp_layer_fwd_fused(plan, q_seq, k_seq, v_seq, o_seq)
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    f0.record()
-    for _ in range(args.steps):
-        basp.basp_layer_fwd_fused(plan, q_seq, k_seq, v_seq, o_seq)
-    f1.record()
-    torch.cuda.synchronize()
-    ms_fused = f0.elapsed_time(f1) / args.steps
-    basp.basp_get_status()
-
-    # the same three launches replayed from a CUDA graph (the calls are capturable: asynchronous, no allocation, no
-    # synchronisation): what the step costs without the host's launch path, which is what config 1 is bound by
-    side = torch.cuda.Stream()
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph, stream=side):
-        step()
-    graph.replay()
-    torch.cuda.synchronize()
-    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    g0.record()
-    for _ in range(args.steps):
-        graph.replay()
-    g1.record()
-    torch.cuda.synchronize()
-    ms_graph = g0.elapsed_time(g1) / args.steps
-    basp.basp_get_status()
-    del graph
-    clocks = sampler.stop() if sampler else None
-
-    # end to end through the C ABI with HOST buffers: H2D of Q, K, V and D2H of O inside the timed region
-    e2e_steps = max(1, min(args.steps, 5))
-    del q_head, k_head, v_head, o_head
-    hq = [t.cpu().pin_memory() for t in q_seq]
-    hk = [t.cpu().pin_memory() for t in k_seq]
-    hv = [t.cpu().pin_memory() for t in v_seq]
-    ho = [torch.empty_like(t).pin_memory() for t in hq]
-    arena = torch.empty(basp.basp_host_arena_bytes(plan), dtype=torch.uint8, device=dev)
-    basp.basp_layer_fwd_host(plan, hq, hk, hv, ho, arena)
-    pdist.barrier()
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        basp.basp_layer_fwd_host(plan, hq, hk, hv, ho, arena)       # synchronises the stream itself
-    torch.cuda.synchronize()
-    e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
-    h2d = sum(t.numel() * 2 for t in hq + hk + hv)
-    d2h = sum(t.numel() * 2 for t in ho)
-
-    ms_per_step = pdist.max_over_ranks(total_ms / args.steps)
-    e2e_ms = pdist.max_over_ranks(e2e_ms)
-    ms_fused_max = pdist.max_over_ranks(ms_fused)
+    # ---- the headline shape: exactly args.steps timed steps after args.warmup untimed ones
+    shape = Shape(basp, w, dev, seed=1000 + rank)
+    t = time_steps(shape, args.steps, args.warmup, rank, local_rank)
+    ms_per_step = pdist.max_over_ranks(t["total_ms"] / args.steps)
+    k = rates(w, t, peaks)
     tokens_all = w.tokens * world
+    fused = None
+    if w.train:
+        e2e_steps = max(1, min(args.steps, 3))
+        e2e_ms = pdist.max_over_ranks(time_e2e_train(shape, e2e_steps, dev))
+        e2e = {"value": tokens_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+               "ms_per_step": e2e_ms, "steps": e2e_steps,
+               "call": "basp_layer_fwd + basp_layer_bwd from device buffers (a training step has no host boundary)"}
+        top, top_name = k["attn_bwd"], "attn_bwd"
+    else:
+        f_ms = pdist.max_over_ranks(time_fused(shape, args.steps, args.warmup))
+        fused = {"ms_per_step": f_ms, "value": tokens_all / (f_ms * 1e-3), "unit": UNIT,
+                 "tflops": w.attn_flops_fwd() / (f_ms * 1e-3) / 1e12, "launches_per_step": 1,
+                 "ms_minus_attention_launch": f_ms - t["ms_attn"]}
+        del shape.q_head, shape.k_head, shape.v_head, shape.o_head
+        e2e_steps = max(1, min(args.steps, 5))
+        e_ms, h2d, d2h = time_e2e_host(shape, e2e_steps, dev)
+        e2e_ms = pdist.max_over_ranks(e_ms)
+        e2e = {"value": tokens_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": e2e_ms, "steps": e2e_steps,
+               "call": "basp_layer_fwd_host (fused kernel per arrived piece of query rows, copies and kernels pipelined, pinned host shards)"}
+        top, top_name = k["attn_fwd"], "attn_fwd"
+    del shape
+    torch.cuda.empty_cache()
+
+    # ---- every benchmark shape under the same clock (one GPU only: the scaling runs stay short)
+    configs = None
+    if world == 1 and not args.no_configs:
+        configs = {}
+        for name in ALL_SHAPES:
+            ww = synth.WORKLOADS[name]
+            configs[name] = measure_shape(basp, ww, dev, rank, local_rank, 3 if ww.train else min(args.steps, 10),
+                                          max(3, min(args.warmup, 5)), peaks)
+    span = measure_span(basp, dev, rank, world, max(2, min(args.steps, 10)), args.warmup) if not args.no_configs else None
 
     if rank == 0:
-        flops = w.attn_flops_fwd()
-        attn_tflops = flops / (ms_attn * 1e-3) / 1e12
-        s2h_gbs = w.reshard_bytes_s2h() / (ms_s2h * 1e-3) / 1e9
-        h2s_gbs = w.reshard_bytes_h2s() / (ms_h2s * 1e-3) / 1e9
         cpu = None
         if world == 1:
-            v, cores, desc, _ = oracle_sample(w)
+            v, cores, desc, _ = oracle_sample(w, budget_rows=2048 if w.train else 8192)
+            if w.train:
+                v, desc = v / 3.5, desc + "; forward sample scaled by 3.5 for forward + backward (4*D + 10*D flop per pair)"
             cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
         line = {
             "metric": METRIC, "value": tokens_all / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": w.name, "N": w.N, "b": w.B, "group_size": K, "S": w.S, "Hq": w.Hq, "Hkv": w.Hkv,
-                       "D": w.D, "causal": True, "path": "reshard_qkv_s2h -> attn_fwd -> reshard_h2s (3 launches/step)",
-                       "l2": "inputs larger than L2 (Q+K+V 768 MiB per step for the default workload)",
-                       "per_gpu_tokens": w.tokens},
-            "clocks": clocks,
-            "e2e": {"value": tokens_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
-                    "call": "basp_layer_fwd_host (fused kernel per arrived piece of query rows, copies and kernels pipelined, pinned host shards)"},
-            "gpu_launches": launches,
-            "ms_per_step_median": statistics.median(per_step), "ms_per_step_best": min(per_step),
-            "roofline": {"kernel": "attn_fwd", "bound": "tensor", "achieved": attn_tflops,
-                         "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
-                         "frac": attn_tflops / peaks["bf16_sustained"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
-                         "peak_source": f"bf16 sustained, of {peaks['source']}", "ms": ms_attn,
-                         "frac_of_burst": attn_tflops / peaks["bf16_burst"], "frac_of_nominal_2250": attn_tflops / 2250.0,
-                         "flops_per_launch": flops},
-            "kernels": {
-                "reshard_qkv_s2h": {"ms": ms_s2h, "bound": "hbm", "achieved": s2h_gbs, "unit": "GB/s",
-                                    "frac": s2h_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": s2h_gbs / 8000.0,
-                                    "bytes": w.reshard_bytes_s2h()},
-                "reshard_h2s": {"ms": ms_h2s, "bound": "hbm", "achieved": h2s_gbs, "unit": "GB/s",
-                                "frac": h2s_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": h2s_gbs / 8000.0,
-                                "bytes": w.reshard_bytes_h2s()},
-            },
-            "fused": {"ms_per_step": ms_fused_max, "value": tokens_all / (ms_fused_max * 1e-3), "unit": UNIT,
-                      "tflops": flops / (ms_fused * 1e-3) / 1e12, "launches_per_step": 1},
-            "graph_replay": {"ms_per_step": ms_graph, "value": w.tokens / (ms_graph * 1e-3), "unit": UNIT,
-                             "what": "the step's three launches captured once into a CUDA graph and replayed"},
-            "cpu_baseline": cpu,
+            "config": config_dict(w), "clocks": t["clocks"], "e2e": e2e, "gpu_launches": t["launches"],
+            "ms_per_step_median": statistics.median(t["per_step"]), "ms_per_step_best": min(t["per_step"]),
+            "roofline": {"kernel": top_name, "bound": "tensor", "achieved": top["tflops"], "peak": peaks["bf16_sustained"],
+                         "unit": "TFLOP/s", "frac": top["frac_of_sustained"], "traffic": ncu_traffic(w.name, top_name),
+                         "peak_source": f"cuBLAS bf16 sustained (the kernel is timed inside a loop), of {peaks['source']}",
+                         "ms": top["ms"], "frac_of_burst": top["frac_of_burst"],
+                         "frac_of_nominal_2250": top["frac_of_nominal_2250"],
+                         "flops_per_launch": w.attn_flops_bwd() if w.train else w.attn_flops_fwd()},
+            "kernels": k, "fused": fused, "configs": configs, "span": span, "cpu_baseline": cpu,
         }
         print(json.dumps(line), flush=True)
     pdist.finalize()
 
 
-def finish_train(args, w, basp, peaks, rank, world, sampler, launches, total_ms, ms_s2h, ms_attn, ms_h2s, ms_bwd, K):
-    """JSON line of a forward + backward workload (BASELINE config 5)."""
-    clocks = sampler.stop() if sampler else None
-    ms_per_step = pdist.max_over_ranks(total_ms / args.steps)
-    tokens_all = w.tokens * world
-    if rank == 0:
-        fwd_tf = w.attn_flops_fwd() / (ms_attn * 1e-3) / 1e12
-        bwd_tf = w.attn_flops_bwd() / (ms_bwd[1] * 1e-3) / 1e12
-        gbs = lambda b, ms: b / (ms * 1e-3) / 1e9
-        cpu = None
-        if world == 1:
-            v, cores, desc, _ = oracle_sample(w, budget_rows=2048)
-            cpu = {"value": v / 3.5, "unit": UNIT, "cores": cores, "kind": "oracle",
-                   "sample": desc + "; forward sample scaled by 3.5 for forward + backward (4*D + 10*D flop per pair)"}
-        line = {
-            "metric": METRIC, "value": tokens_all / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": w.name, "N": w.N, "b": w.B, "group_size": K, "S": w.S, "Hq": w.Hq, "Hkv": w.Hkv,
-                       "D": w.D, "causal": True,
-                       "path": "forward (s2h, attn_fwd, h2s) + backward (s2h dO, attn_bwd, h2s dQ/dK/dV)",
-                       "l2": "inputs larger than L2", "per_gpu_tokens": w.tokens},
-            "clocks": clocks, "e2e": None, "gpu_launches": launches,
-            "roofline": {"kernel": "attn_bwd (memset + Delta + main + dQ conversion)", "bound": "tensor",
-                         "achieved": bwd_tf, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
-                         "frac": bwd_tf / peaks["bf16_sustained"], "traffic": None,
-                         "peak_source": f"bf16 sustained, of {peaks['source']}", "ms": ms_bwd[1],
-                         "frac_of_burst": bwd_tf / peaks["bf16_burst"], "frac_of_nominal_2250": bwd_tf / 2250.0,
-                         "flops_per_launch": w.attn_flops_bwd()},
-            "kernels": {
-                "attn_fwd": {"ms": ms_attn, "bound": "tensor", "achieved": fwd_tf, "unit": "TFLOP/s",
-                             "frac": fwd_tf / peaks["bf16_sustained"]},
-                "reshard_qkv_s2h": {"ms": ms_s2h, "achieved": gbs(w.reshard_bytes_s2h(), ms_s2h), "unit": "GB/s",
-                                    "frac": gbs(w.reshard_bytes_s2h(), ms_s2h) / peaks["hbm_gbs"]},
-                "reshard_h2s_o": {"ms": ms_h2s, "achieved": gbs(w.reshard_bytes_h2s(), ms_h2s), "unit": "GB/s",
-                                  "frac": gbs(w.reshard_bytes_h2s(), ms_h2s) / peaks["hbm_gbs"]},
-                "reshard_s2h_do": {"ms": ms_bwd[0], "achieved": gbs(w.reshard_bytes_h2s(), ms_bwd[0]), "unit": "GB/s",
-                                   "frac": gbs(w.reshard_bytes_h2s(), ms_bwd[0]) / peaks["hbm_gbs"]},
-                "reshard_grads_h2s": {"ms": ms_bwd[2], "achieved": gbs(w.reshard_bytes_s2h(), ms_bwd[2]), "unit": "GB/s",
-                                      "frac": gbs(w.reshard_bytes_s2h(), ms_bwd[2]) / peaks["hbm_gbs"]},
-            },
-            "cpu_baseline": cpu,
-        }
-        print(json.dumps(line), flush=True)
-    pdist.finalize()
+def time_projections(basp, shape: Shape, args, dev):
+    """The projections on either side of the core (not part of the step): X W_qkv^T (plain and with the rotary
+    embedding in its epilogue) and O W_o^T."""
+    w, plan = shape.w, shape.plan
+    N, T, Bl = w.N, plan.T, plan.Bl
+    hidden = w.Hq * w.D
+    xs = [shape.randn((Bl * T, hidden)) for _ in range(N)]
+    w_qkv = (torch.randn(((w.Hq + 2 * w.Hkv) * w.D, hidden), device=dev) / hidden ** 0.5).to(torch.bfloat16)
+    w_o = (torch.randn((hidden, w.Hq * w.D), device=dev) / hidden ** 0.5).to(torch.bfloat16)
+    ys = [torch.empty((Bl * T, hidden), dtype=torch.bfloat16, device=dev) for _ in range(N)]
+    pe = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    for it in range(args.warmup + args.steps):
+        if it == args.warmup:
+            pe[0].record()
+        basp.basp_qkv_proj(plan, hidden, xs, w_qkv, shape.q_seq, shape.k_seq, shape.v_seq)
+    pe[1].record()
+    for it in range(args.steps):
+        basp.basp_out_proj(plan, hidden, shape.o_seq, w_o, ys)
+    pe[2].record()
+    ms_rope = None
+    if w.D in (64, 128):
+        cos, sin = (t.t().contiguous().to(dev) for t in synth.rope_tables(w.S, w.D))      # feature-major
+        re = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        for it in range(args.warmup + args.steps):
+            if it == args.warmup:
+                re[0].record()
+            basp.basp_qkv_proj_rope(plan, hidden, xs, w_qkv, cos, sin, shape.q_seq, shape.k_seq, shape.v_seq)
+        re[1].record()
+        torch.cuda.synchronize()
+        ms_rope = re[0].elapsed_time(re[1]) / args.steps
+    torch.cuda.synchronize()
+    basp.basp_get_status()
+    ms_qkv, ms_out = pe[0].elapsed_time(pe[1]) / args.steps, pe[1].elapsed_time(pe[2]) / args.steps
+    f_qkv = 2.0 * N * Bl * T * hidden * (w.Hq + 2 * w.Hkv) * w.D
+    f_out = 2.0 * N * Bl * T * hidden * w.Hq * w.D
+    return {"hidden": hidden, "qkv_ms": ms_qkv, "qkv_tflops": f_qkv / ms_qkv / 1e9, "out_ms": ms_out,
+            "out_tflops": f_out / ms_out / 1e9, "qkv_rope_ms": ms_rope,
+            "qkv_rope_tflops": f_qkv / ms_rope / 1e9 if ms_rope else None}
 
 
 def main():
@@ -455,7 +579,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="basp", choices=["basp", "reference"])
     ap.add_argument("--proj", action="store_true", help="also time the QKV and output projection GEMMs (with --quick)")
-    ap.add_argument("--quick", action="store_true", help="time the three kernels only (for profiler runs)")
+    ap.add_argument("--quick", action="store_true", help="time the kernels of one shape only (for profiler runs)")
+    ap.add_argument("--no-configs", action="store_true", help="the headline shape only (no `configs`, no `span`)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     w = synth.WORKLOADS[args.workload]

@@ -27,7 +27,9 @@
  *   - "*_shards" arguments are HOST arrays of n_ranks DEVICE pointers; the array is read
  *     during the call and not retained; every device pointer must be 16-byte aligned;
  *   - the caller owns every device buffer (workspace included); the library allocates no
- *     device memory and keeps no pointer after return; the plan is the only library object;
+ *     device memory and keeps no pointer after return; the plan is the only library object
+ *     (one exception, stated there: basp_layer_fwd_static keeps its scratch in a fixed array
+ *     inside the library's device image and remembers that array's address per device);
  *   - launches are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = the
  *     default stream); no call synchronises the device except basp_get_status and
  *     basp_layer_fwd_host;
@@ -161,7 +163,7 @@ int basp_reshard_qkv_s2h(const basp_plan *plan, const void *const *q_seq, const 
  *   O[i] = sum_{j visible} softmax_j(scale * q_i . k_j) v_j,   LSE[i] = ln sum_j exp(scale * q_i . k_j)
  * Inputs/outputs are HEAD-sharded; lse_shards may be NULL (then no LSE is written), else a
  * host array of n_ranks device pointers to fp32 [Bl][Hq/K][S].  softmax_scale = 0 selects
- * 1/sqrt(D).  bf16 operands, fp32 accumulation and softmax, P rounded to bf16 before P.V.
+ * 1/sqrt(D); a negative, infinite or NaN scale is BASP_ERR_INVALID in every call that takes one.  bf16 operands, fp32 accumulation and softmax, P rounded to bf16 before P.V.
  * Requires D a multiple of 16 up to 128 (else BASP_ERR_UNSUPPORTED; the kernels are 64 and 128 columns wide, for a
  * D in between the tile loads zero-fill the missing columns); S is arbitrary (a ragged last tile is masked).
  * A bounded wait that expires inside the kernel is reported by basp_get_status. */
@@ -189,12 +191,16 @@ size_t basp_workspace_bytes(const basp_plan *plan);
  * or other allocating routine; inputs and outputs are still the caller's.
  *   - Plans whose basp_workspace_bytes exceeds BASP_STATIC_SCRATCH_BYTES are refused with
  *     BASP_ERR_WORKSPACE (basp_last_cuda_error then names both sizes).
- *   - The first call on each device looks up the array's device address (one runtime query, made
- *     with that device current); make that first call before starting any stream capture.
+ *   - The first call on each device is the set-up call: it looks up the array's device address (one
+ *     runtime query, made with that device current), and if nothing of this library's device code
+ *     has run on that device before, that is also when the CUDA runtime loads the library's image and
+ *     the GPU commits the array's memory.  Make that first call at start-up: before the device's
+ *     memory is handed to another pool, and before starting any stream capture.  Later calls leave
+ *     the amount of free device memory exactly as they found it.
  *   - All calls on a device share the one array.  It keeps whatever the last call wrote; nothing
  *     needs clearing because each call overwrites every byte it later reads.  Two calls that can
  *     overlap on the GPU (different streams, no dependency) race on it: serialise them.
- * Results are identical to basp_layer_fwd. */
+ * Results are bit-identical to basp_layer_fwd's (the same launches on the same inputs). */
 #define BASP_STATIC_SCRATCH_BYTES (16u << 20)
 int basp_layer_fwd_static(const basp_plan *plan, const void *const *q_seq, const void *const *k_seq,
                           const void *const *v_seq, void *const *o_seq, float *const *lse_shards,
@@ -238,9 +244,9 @@ int basp_layer_fwd_fused_ranks(const basp_plan *plan, const void *const *q_seq, 
                                const void *const *v_seq, void *const *o_seq, float *const *lse_shards,
                                float softmax_scale, int rank_begin, int rank_count, void *stream);
 
-/* After basp_layer_fwd (or basp_layer_fwd_static) returns, the workspace holds the head-sharded
- * Q, K, V and O of every rank; this call writes their addresses (n_ranks pointers each) so that a
- * training step can keep them for the backward pass instead of resharding again. */
+/* After basp_layer_fwd returns, the workspace holds the head-sharded Q, K, V and O of every rank; this call
+ * writes their addresses (n_ranks pointers each) so that a training step can keep them for the backward pass
+ * instead of resharding again.  (The fixed array of basp_layer_fwd_static cannot be reached from outside.) */
 int basp_layer_workspace_shards(const basp_plan *plan, void *workspace, void **q_head, void **k_head,
                                 void **v_head, void **o_head);
 
@@ -251,9 +257,12 @@ int basp_layer_workspace_shards(const basp_plan *plan, void *workspace, void **q
  * with dK, dV summed over the Hq/Hkv query heads of a KV head.  All operands HEAD-sharded: q, o, do, dq
  * [Bl][S][Hq/K][D]; k, v, dk, dv [Bl][S][Hkv/K][D]; lse as written by the forward.  bf16 in and out,
  * fp32 accumulation; dQ is accumulated with floating-point atomics, so its last bits may differ
- * between runs.  Requires D a multiple of 16 up to 128 (the kernel is 128 columns wide: a smaller D runs with the
- * missing columns zero-filled by the tile loads and costs the same time as D = 128); S is arbitrary (ragged last tiles are masked).  `workspace`: device memory of at least
- * basp_attn_bwd_workspace_bytes(plan) bytes (fp32 dQ accumulator and Delta). */
+ * between runs.  Requires D a multiple of 16 up to 128 (two kernels, 64 and 128 columns wide; a D in between runs on
+ * the wider one with the missing columns zero-filled by the tile loads); S is arbitrary (ragged last tiles are masked).
+ * `workspace`: device memory of at least basp_attn_bwd_workspace_bytes(plan) bytes (fp32 dQ accumulator, Delta and a
+ * few counters).  For long causal sequences at D > 64 the thread blocks that work on one (rank, sequence, KV head)
+ * start their sweeps together (they wait for one another inside the launch, every wait bounded), so that launch is
+ * made cooperatively; where the device cannot hold all of its blocks at once the ordinary schedule runs instead. */
 int basp_attn_bwd(const basp_plan *plan, const void *const *q_head, const void *const *k_head,
                   const void *const *v_head, const void *const *o_head, const void *const *do_head,
                   const float *const *lse_shards, void *const *dq_head, void *const *dk_head,
@@ -262,8 +271,8 @@ int basp_attn_bwd(const basp_plan *plan, const void *const *q_head, const void *
 size_t basp_attn_bwd_workspace_bytes(const basp_plan *plan);
 /* The same gradients, bit-identical from run to run: two passes (dK and dV with the key tile resident, dQ with the
  * query tile resident) instead of one pass that adds dQ partial sums into a global accumulator in whatever order the
- * thread blocks finish.  Costs the scores and the element-wise part twice (measured about 7 % slower on the config 5
- * shape); same arguments, workspace and errors as basp_attn_bwd. */
+ * thread blocks finish.  Costs the scores and the element-wise part twice (slower than the one-pass form); same
+ * arguments, workspace and errors as basp_attn_bwd. */
 int basp_attn_bwd_deterministic(const basp_plan *plan, const void *const *q_head, const void *const *k_head,
                                 const void *const *v_head, const void *const *o_head, const void *const *do_head,
                                 const float *const *lse_shards, void *const *dq_head, void *const *dk_head,

@@ -8,7 +8,7 @@ The forward keeps its workspace (head-sharded Q, K, V, O) and the log-sum-exp fo
 paper's setting does between the two passes; the backward needs a second workspace (basp_layer_bwd_workspace_bytes).
 Both are allocated through torch's caching allocator on the current device.  With fused=True the forward is the one
 fused kernel and keeps nothing but its output and the log-sum-exp (no head-sharded copies live between the passes: for
-config 5 that is 2.5 GiB less); the backward then redoes the exchanges of Q, K, V and O itself.
+the 128K-token training shape that is 2.5 GiB less); the backward then redoes the exchanges of Q, K, V and O itself.
 """
 from __future__ import annotations
 

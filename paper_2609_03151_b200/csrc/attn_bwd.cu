@@ -324,6 +324,7 @@ int bwd_entry(const basp_plan *pl, const void *const *q_head, const void *const 
     if (!pl || !q_head || !k_head || !v_head || !o_head || !do_head || !lse_shards || !dq_head || !dk_head ||
         !dv_head || !workspace)
         return BASP_ERR_NULL;
+    if (!scale_ok(softmax_scale)) return BASP_ERR_INVALID;
     if (pl->D < 16 || pl->D > 128 || pl->D % 16 != 0) return BASP_ERR_UNSUPPORTED;
     if (!aligned16(workspace)) return BASP_ERR_ALIGN;
     if (workspace_bytes < basp_attn_bwd_workspace_bytes(pl)) return BASP_ERR_WORKSPACE;

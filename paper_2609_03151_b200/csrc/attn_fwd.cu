@@ -19,9 +19,7 @@
 
 int *basp_status_device_ptr();
 
-#ifndef BASP_BAND_TARGET
-#define BASP_BAND_TARGET 32   // CTAs that share one KV stream at a time (query blocks per band x query heads per KV head)
-#endif
+constexpr int kBandTarget = 32;   // CTAs that share one KV stream at a time (query blocks per band x query heads per KV head)
 
 namespace {
 
@@ -52,7 +50,7 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
     {
         const int q_per_kv = pl->Hq_l / pl->Hkv_l;
         prm.r_begin = range[0]; prm.r_count = range[1]; prm.qb_begin = range[2]; prm.qb_count = range[3];
-        int band = BASP_BAND_TARGET / q_per_kv < 1 ? 1 : (BASP_BAND_TARGET / q_per_kv > 16 ? 16 : BASP_BAND_TARGET / q_per_kv);
+        int band = kBandTarget / q_per_kv < 1 ? 1 : (kBandTarget / q_per_kv > 16 ? 16 : kBandTarget / q_per_kv);
         while (prm.qb_count % band != 0) --band;
         prm.qb_band = band;
         prm.div_per_band = make_fastdiv((uint32_t)(range[1] * pl->Bl * pl->Hq_l * band));
@@ -100,6 +98,9 @@ int basp_attn_dispatch_range(const basp_plan *pl, const void *const *q, const vo
                              void *const *o, float *const *lse, float scale, bool fused, const int *range,
                              void *stream, bool cta_per_item) {
     if (!pl || !q || !k || !v || !o) return BASP_ERR_NULL;
+    // the kernel takes the row maximum of the raw scores and masks with -inf before it scales: a negative scale would pick
+    // the wrong reference and turn masked keys into +inf
+    if (!scale_ok(scale)) return BASP_ERR_INVALID;
     if (pl->D < 16 || pl->D > 128 || pl->D % 16 != 0) return BASP_ERR_UNSUPPORTED;
     if (fused && pl->T % kTile != 0) return BASP_ERR_UNSUPPORTED;
     // A short last shard (K does not divide S) holds its sequences T_last rows apart, the others T: the kernel's tile

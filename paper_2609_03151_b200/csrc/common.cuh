@@ -37,3 +37,5 @@ __device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv &f) {
 }
 
 static inline bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
+// A softmax scale the kernels accept: 0 (= 1/sqrt(D)) or a positive finite number (not NaN, not negative, not infinite).
+static inline bool scale_ok(float s) { return s >= 0.f && s <= 3.0e38f; }

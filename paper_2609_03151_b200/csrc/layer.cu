@@ -34,6 +34,7 @@ extern "C" int basp_layer_fwd(const basp_plan *p, const void *const *q_seq, cons
                               const void *const *v_seq, void *const *o_seq, float *const *lse_shards,
                               void *workspace, size_t workspace_bytes, float softmax_scale, void *stream) {
     if (!p || !workspace) return BASP_ERR_NULL;
+    if (!scale_ok(softmax_scale)) return BASP_ERR_INVALID;
     if (!aligned16(workspace)) return BASP_ERR_ALIGN;
     if (workspace_bytes < basp_workspace_bytes(p)) return BASP_ERR_WORKSPACE;
     char *w = (char *)workspace;
@@ -78,6 +79,7 @@ extern "C" int basp_layer_bwd(const basp_plan *p, const void *const *q_head, con
                               void *const *dv_seq, void *workspace, size_t workspace_bytes, float softmax_scale,
                               void *stream) {
     if (!p || !workspace) return BASP_ERR_NULL;
+    if (!scale_ok(softmax_scale)) return BASP_ERR_INVALID;
     if (!aligned16(workspace)) return BASP_ERR_ALIGN;
     if (workspace_bytes < basp_layer_bwd_workspace_bytes(p)) return BASP_ERR_WORKSPACE;
     char *w = (char *)workspace;
@@ -110,6 +112,7 @@ extern "C" int basp_layer_bwd_seq(const basp_plan *p, const void *const *q_seq, 
                                   void *const *dv_seq, void *workspace, size_t workspace_bytes, float softmax_scale,
                                   void *stream) {
     if (!p || !workspace) return BASP_ERR_NULL;
+    if (!scale_ok(softmax_scale)) return BASP_ERR_INVALID;
     if (!aligned16(workspace)) return BASP_ERR_ALIGN;
     if (workspace_bytes < basp_layer_bwd_seq_workspace_bytes(p)) return BASP_ERR_WORKSPACE;
     char *w = (char *)workspace;
@@ -202,6 +205,7 @@ extern "C" int basp_layer_fwd_host(const basp_plan *p, const void *const *q_seq_
                                    const void *const *v_seq_host, void *const *o_seq_host, void *device_arena,
                                    size_t arena_bytes, float softmax_scale, void *stream) {
     if (!p || !q_seq_host || !k_seq_host || !v_seq_host || !o_seq_host || !device_arena) return BASP_ERR_NULL;
+    if (!scale_ok(softmax_scale)) return BASP_ERR_INVALID;
     if (!aligned16(device_arena)) return BASP_ERR_ALIGN;
     if (arena_bytes < basp_host_arena_bytes(p)) return BASP_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;

@@ -168,12 +168,15 @@ int fill_tensor(const basp_plan *p, const TensorArg &a, bool to_head, int r_begi
         if ((need_seq && !a.seq[r]) || (need_head && !a.head[r])) return BASP_ERR_NULL;
         if ((need_seq && !aligned16(a.seq[r])) || (need_head && !aligned16(a.head[r]))) return BASP_ERR_ALIGN;
     }
-    // out-of-place only: no destination shard may overlap a source shard
+    // out-of-place only: no destination shard may overlap a source shard.  The head side's extent is exact (whole
+    // sequences of S tokens: smaller than Bl*T*H*D where the group size does not divide S), so a buffer that starts
+    // right behind the last head shard is not taken for an overlap.
+    const size_t head_extent = (size_t)p->Bl * p->S * (rep > 1 ? (size_t)1 : (size_t)(a.n_heads / p->K)) * p->D * 2;
     for (int i = r_begin; i < r_begin + r_count; ++i)
         for (int j = g_begin; j < g_end; ++j) {
             const char *s = t->seq[i], *d = t->head[j];
             const size_t seq_bytes = shard_bytes / p->T * basp_rank_tokens(p, i % p->K);
-            if (s < d + head_bytes && d < s + seq_bytes) return BASP_ERR_ALIAS;
+            if (s < d + head_extent && d < s + seq_bytes) return BASP_ERR_ALIAS;
         }
     t->rep = (uint32_t)rep;
     t->run_v = (uint32_t)(run_bytes / 16);

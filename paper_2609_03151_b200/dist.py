@@ -101,23 +101,45 @@ def shard_addresses(buffer_ptrs, n_ranks: int, shard_bytes: int, offset: int = 0
     return [int(buffer_ptrs[r // per]) + offset + (r % per) * shard_bytes for r in range(n_ranks)]
 
 
-class SymmetricShards:
-    """One symmetric-memory buffer per GPU holding this GPU's shards of several tensors, mapped into every process of
-    the group (torch symmetric memory over NVLink).  `tensors` = {name: shard_bytes}.  Needs an initialised NCCL
-    process group with one process per GPU."""
+def _symmetric_allocator(nbytes: int, group):
+    """Default allocator of SymmetricShards: torch symmetric memory (every process maps every GPU's buffer), or, for a
+    single process, an ordinary device buffer (there is no peer to map)."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size(group) == 1:
+        buf = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        return buf, [buf.data_ptr()]
+    import torch.distributed._symmetric_memory as symm_mem
+    buf = symm_mem.empty(nbytes, dtype=torch.uint8, device=dev)
+    handle = symm_mem.rendezvous(buf, group)
+    buf._basp_symm_handle = handle          # keeps the mapping alive as long as the buffer
+    return buf, [int(p) for p in handle.buffer_ptrs]
 
-    def __init__(self, n_ranks: int, tensors: dict, group=None):
-        import torch.distributed._symmetric_memory as symm_mem
-        self.group = group if group is not None else dist.group.WORLD
-        self.world, self.gpu = dist.get_world_size(self.group), dist.get_rank(self.group)
+
+class SymmetricShards:
+    """One buffer per GPU holding this GPU's shards of several tensors, mapped into every process of the group (torch
+    symmetric memory over NVLink).  `tensors` = {name: shard_bytes}.  With more than one process it needs an
+    initialised NCCL process group with one process per GPU.  `allocator(nbytes, group) -> (buffer, base addresses of
+    every GPU's buffer as mapped here)` replaces the symmetric-memory allocation (tests of the layout arithmetic run on
+    CPU with it); `world` / `gpu` default to the process group's size and this process's rank."""
+
+    def __init__(self, n_ranks: int, tensors: dict, group=None, allocator=None, world: int | None = None,
+                 gpu: int | None = None):
+        initialised = dist.is_available() and dist.is_initialized()
+        self.group = group if group is not None else (dist.group.WORLD if initialised else None)
+        self.world = world if world is not None else (dist.get_world_size(self.group) if initialised else 1)
+        self.gpu = gpu if gpu is not None else (dist.get_rank(self.group) if initialised else 0)
         self.n_ranks, self.local = n_ranks, ranks_of_gpu(n_ranks, self.world, self.gpu)
         self.layout, off = {}, 0
         for name, shard_bytes in tensors.items():
+            if int(shard_bytes) % 16:
+                raise ValueError("shards must stay 16-byte aligned")
             self.layout[name] = (off, int(shard_bytes))
             off += (len(self.local) * int(shard_bytes) + 255) // 256 * 256
-        self.buffer = symm_mem.empty(off, dtype=torch.uint8, device=torch.device("cuda", torch.cuda.current_device()))
-        self.handle = symm_mem.rendezvous(self.buffer, self.group)
-        self.buffer_ptrs = [int(p) for p in self.handle.buffer_ptrs]
+        self.nbytes = off
+        self.buffer, ptrs = (allocator or _symmetric_allocator)(off, self.group)
+        self.buffer_ptrs = [int(p) for p in ptrs]
+        if len(self.buffer_ptrs) != self.world:
+            raise ValueError("the allocator must return one base address per GPU")
 
     def addresses(self, name: str) -> list[int]:
         off, shard_bytes = self.layout[name]
@@ -131,20 +153,65 @@ class SymmetricShards:
             raise ValueError("rank lives on another GPU")
         return self.buffer[off + i * shard_bytes: off + (i + 1) * shard_bytes]
 
+    def remote_fraction(self, group_size: int) -> float:
+        """Share of a rank's exchange partners that live on another GPU: 1 - min(ranks per GPU, K) / K (what crosses
+        NVLink of the bytes that the all-to-alls of a K-rank group move)."""
+        return 1.0 - min(len(self.local), group_size) / float(group_size)
 
-def layer_fwd_fused_multi_gpu(plan, shards: "SymmetricShards", softmax_scale: float = 0.0, stream=None):
+
+def _group_barrier(group):
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier(group)
+
+
+def _resolve_stream(stream):
+    return stream if stream is not None else torch.cuda.current_stream()
+
+
+def layer_fwd_fused_multi_gpu(plan, shards: "SymmetricShards", softmax_scale: float = 0.0, stream=None, binding=None,
+                              barrier=None, lse=None):
     """The layer when a group spans GPUs: every GPU runs the fused kernel for its own ranks over the group's
     sequence shards (`shards` holds tensors "q", "k", "v", "o").  The kernels never wait for one another: the two
     host barriers order the GPUs (inputs complete before anyone reads them, nobody reuses a buffer before all are
-    done)."""
-    from . import binding
-    torch.cuda.current_stream().synchronize()
-    dist.barrier(shards.group)
+    done), and both follow a synchronisation of the SAME stream the kernel is launched on.  `binding` and `barrier`
+    default to the CUDA binding and the process group's barrier (tests pass stand-ins)."""
+    if binding is None:
+        from . import binding
+    barrier = barrier or (lambda: _group_barrier(shards.group))
+    s = _resolve_stream(stream)
+    s.synchronize()
+    barrier()
     binding.basp_layer_fwd_fused_ranks(plan, shards.addresses("q"), shards.addresses("k"), shards.addresses("v"),
-                                       shards.addresses("o"), shards.local.start, len(shards.local),
-                                       softmax_scale=softmax_scale, stream=stream)
-    torch.cuda.current_stream().synchronize()
-    dist.barrier(shards.group)
+                                       shards.addresses("o"), shards.local.start, len(shards.local), lse_shards=lse,
+                                       softmax_scale=softmax_scale, stream=s)
+    s.synchronize()
+    barrier()
+
+
+def layer_fwd_three_step_multi_gpu(plan, shards: "SymmetricShards", softmax_scale: float = 0.0, stream=None,
+                                   binding=None, barrier=None, lse=None):
+    """The same layer as three exchanges-and-kernels, for comparison with the fused form: push this GPU's sequence
+    shards of Q, K, V into the head shards of its groups' members ("qh", "kh", "vh"; remote members over NVLink),
+    attention over its own head shards, pull its sequence shards of O out of the group's "oh".  A host barrier after
+    each step: a step reads what other GPUs wrote in the step before."""
+    if binding is None:
+        from . import binding
+    barrier = barrier or (lambda: _group_barrier(shards.group))
+    s = _resolve_stream(stream)
+    r0, cnt = shards.local.start, len(shards.local)
+    a = shards.addresses
+    s.synchronize()
+    barrier()
+    binding.basp_reshard_qkv_s2h_ranks(plan, a("q"), a("k"), a("v"), a("qh"), a("kh"), a("vh"), r0, cnt, stream=s)
+    s.synchronize()
+    barrier()
+    binding.basp_attn_fwd_ranks(plan, a("qh"), a("kh"), a("vh"), a("oh"), r0, cnt, lse_shards=lse,
+                                softmax_scale=softmax_scale, stream=s)
+    s.synchronize()
+    barrier()
+    binding.basp_reshard_h2s_ranks(plan, plan.Hq, a("oh"), a("o"), r0, cnt, stream=s)
+    s.synchronize()
+    barrier()
 
 
 def finalize():

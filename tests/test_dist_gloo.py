@@ -122,3 +122,101 @@ def test_ranks_of_gpu_and_addresses():
         assert False
     except ValueError:
         pass
+
+
+def _cpu_allocator(world, gpu, base=0x7000_0000_0000):
+    """Stand-in for symmetric memory: a host buffer and invented base addresses, one per 'GPU' (1 TiB apart)."""
+    def alloc(nbytes, group):
+        buf = torch.zeros(nbytes, dtype=torch.uint8)
+        return buf, [base + g * (1 << 40) for g in range(world)]
+    return alloc
+
+
+def test_symmetric_shards_layout_on_cpu():
+    """Layout arithmetic of the per-GPU shard buffer: tensors back to back (256-byte aligned blocks), this GPU's ranks
+    consecutive inside each block, the same offsets on every GPU."""
+    n_ranks, world, gpu = 8, 4, 2
+    sizes = {"q": 4096, "k": 1040, "v": 1040, "o": 4096}          # 1040: a block that needs padding to 256
+    sh = pdist.SymmetricShards(n_ranks, sizes, allocator=_cpu_allocator(world, gpu), world=world, gpu=gpu)
+    assert list(sh.local) == [4, 5]
+    offs = {"q": 0, "k": 8192, "v": 8192 + 2304, "o": 8192 + 2 * 2304}
+    assert sh.nbytes == offs["o"] + 8192
+    base = lambda g: 0x7000_0000_0000 + g * (1 << 40)
+    for name, sz in sizes.items():
+        assert sh.addresses(name) == [base(r // 2) + offs[name] + (r % 2) * sz for r in range(n_ranks)]
+        assert all(a % 16 == 0 for a in sh.addresses(name))
+    sh.local_shard("k", 5)[:] = 7
+    assert int(sh.buffer[offs["k"] + 1040: offs["k"] + 2080].sum()) == 7 * 1040 and int(sh.buffer.sum()) == 7 * 1040
+    for bad in (3, 6):
+        try:
+            sh.local_shard("k", bad)
+            assert False
+        except ValueError:
+            pass
+    assert sh.remote_fraction(8) == 0.75 and sh.remote_fraction(2) == 0.0 and sh.remote_fraction(4) == 0.5
+    try:
+        pdist.SymmetricShards(n_ranks, {"q": 24}, allocator=_cpu_allocator(world, gpu), world=world, gpu=gpu)
+        assert False
+    except ValueError:
+        pass
+
+
+class _RecordingStream:
+    def __init__(self, log, name):
+        self.log, self.name = log, name
+
+    def synchronize(self):
+        self.log.append(("sync", self.name))
+
+
+def _worker_multi_gpu_order(rank, world, port, out_dir):
+    """Host ordering of the group-spanning layer (synchronise the launch stream, barrier, launch, synchronise the same
+    stream, barrier) with the oracle standing in for the kernel: each process produces only its ranks' output shards
+    and the union is the whole layer."""
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    pdist.init(backend="gloo")
+    wl = synth.Workload("g", N=4, B=1, S=64, Hq=4, Hkv=2, D=8)             # one group of 4 ranks over 2 'GPUs'
+    Xq, Xk, Xv = (synth.bits(t) for t in synth.make_qkv(wl, seed=3))
+    pl = oracle.plan(wl.N, wl.B, wl.S)
+    ref = oracle.layer_fwd(Xq, Xk, Xv, pl)
+    shard_bytes = {"q": pl.T * wl.Hq * wl.D * 2, "k": pl.T * wl.Hkv * wl.D * 2, "v": pl.T * wl.Hkv * wl.D * 2,
+                   "o": pl.T * wl.Hq * wl.D * 2}
+    sh = pdist.SymmetricShards(wl.N, shard_bytes, allocator=_cpu_allocator(world, rank), world=world, gpu=rank)
+    log, produced = [], {}
+
+    class StubBinding:
+        @staticmethod
+        def basp_layer_fwd_fused_ranks(plan, q, k, v, o, rank_begin, rank_count, lse_shards=None, softmax_scale=0.0,
+                                       stream=None):
+            log.append(("launch", stream.name, rank_begin, rank_count))
+            assert q == sh.addresses("q") and o == sh.addresses("o") and len(q) == wl.N
+            for r in range(rank_begin, rank_begin + rank_count):
+                produced[r] = ref["o_seq"][r]
+
+    def barrier():
+        log.append(("barrier",))
+        dist.barrier()
+
+    side = _RecordingStream(log, "side")
+    pdist.layer_fwd_fused_multi_gpu("plan", sh, stream=side, binding=StubBinding, barrier=barrier)
+    mine = pdist.ranks_of_gpu(wl.N, world, rank)
+    assert log == [("sync", "side"), ("barrier",), ("launch", "side", mine.start, len(mine)), ("sync", "side"), ("barrier",)]
+    assert sorted(produced) == list(mine)
+    gathered = [None] * world
+    dist.all_gather_object(gathered, {r: a for r, a in produced.items()})
+    union = {}
+    for d in gathered:
+        assert not (set(d) & set(union))
+        union.update(d)
+    got = oracle.gather(np.stack([union[r] for r in range(wl.N)]), pl)
+    full, _ = oracle.attn_fwd(Xq, Xk, Xv)
+    assert np.array_equal(got, full)
+    pdist.finalize()
+    open(os.path.join(out_dir, f"order{rank}"), "w").write("ok")
+
+
+def test_two_process_multi_gpu_layer_ordering(tmp_path):
+    port = _free_port()
+    mp.spawn(_worker_multi_gpu_order, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    assert all((tmp_path / f"order{r}").exists() for r in range(2))

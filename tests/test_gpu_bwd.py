@@ -59,7 +59,7 @@ def run_attn_bwd(basp, w, causal=True, seed=0, deterministic=False):
     ("llama_T128", synth.shrink(synth.WORKLOADS["llama3_8b_128k_train"], 128)),
     ("llama_b2_T256", synth.shrink(synth.WORKLOADS["llama3_8b_32k"], 256)),
     ("ulysses", synth.Workload("ulysses", N=4, B=2, S=512, Hq=8, Hkv=4, D=128, G=1)),
-    ("head_dim_64_config1", synth.WORKLOADS["tiny"]),                                        # BASELINE config 1
+    ("head_dim_64_tiny", synth.WORKLOADS["tiny"]),                                           # N=4, b=2, S=1024, 8 heads of 64
     ("head_dim_96", synth.Workload("d96", N=2, B=1, S=512, Hq=4, Hkv=2, D=96)),             # hidden 3072 / 32 heads
     ("head_dim_80", synth.shrink(synth.WORKLOADS["t2_qwen25_3b"], 128)),                    # hidden 2560 / 32 heads
     ("head_dim_48", synth.Workload("d48", N=2, B=2, S=256, Hq=2, Hkv=1, D=48)),

@@ -47,7 +47,7 @@ def test_layer_matches_oracle(basp, w, fused):
 
 
 def test_tiny_basp_equals_ulysses_equals_unpartitioned(basp):
-    """BASELINE config 1: b=2 (two groups of 2) vs b-agnostic Ulysses (one group of 4) vs no partition.
+    """The tiny layer (N=4, S=1024, 8 heads of 64): b=2 (two groups of 2) vs b-agnostic Ulysses (one group of 4) vs no partition.
     The per-row tile schedule does not depend on the grouping, so the GPU outputs agree bit for bit."""
     w = synth.WORKLOADS["tiny"]
     Xq, Xk, Xv, op = oracle_inputs(w)
@@ -87,7 +87,7 @@ def test_host_buffer_entry(basp, w, causal):
 
 @pytest.mark.parametrize("name", ["llama3_8b_32k", "sweep_b1"])
 def test_host_buffer_entry_full_size_sampled_rows(basp, name):
-    """The host-buffer entry at full size, in both orders of its pipeline (config 2: the link is the longer side; config 3
+    """The host-buffer entry at full size, in both orders of its pipeline (Llama-3-8B shape at 32K with b = 2: the link is the longer side; 64K
     at b = 1: the GPU is), on sampled output rows."""
     w = synth.WORKLOADS[name]
     q, k, v = synth.make_qkv(w, seed=0)

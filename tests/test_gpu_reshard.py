@@ -83,7 +83,7 @@ def test_arena_slices_and_guard_bands(basp):
 @pytest.mark.parametrize("name", ["llama3_8b_32k", "sweep_b1", "sweep_b4", "sweep_b8", "qwen25_7b_64k",
                                   "llama3_8b_128k_train"])
 def test_full_size_reshard_sampled(basp, name):
-    """BASELINE configs 2 to 5 at full size (the launches the benchmark times): the closed-form
+    """The benchmark shapes from 32K to 128K tokens at full size (the launches the benchmark times): the closed-form
     destination of sampled source runs, plus the round trip being the identity."""
     w = synth.WORKLOADS[name]
     pl = basp.basp_plan_create(w.N, w.B, w.S, w.Hq, w.Hkv, w.D)
@@ -103,3 +103,25 @@ def test_full_size_reshard_sampled(basp, name):
     torch.cuda.synchronize()
     for a, b in zip(seq, back):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("name", ["llama3_8b_32k", "qwen25_7b_64k"])
+def test_full_size_three_tensor_exchange_against_oracle(basp, name):
+    """The launches the benchmark times, at full size and on every element: Q, K and V through the one-launch first
+    exchange (basp_reshard_qkv_s2h) and O through the reverse one, bit for bit against the oracle's index loops."""
+    w = synth.WORKLOADS[name]
+    pl = basp.basp_plan_create(w.N, w.B, w.S, w.Hq, w.Hkv, w.D)
+    op = oracle.plan(w.N, w.B, w.S)
+    seq = [synth.random_bits((w.N, 1, pl.T, h, w.D), seed=i) for i, h in enumerate((w.Hq, w.Hkv, w.Hkv))]
+    src = [to_dev(a) for a in seq]
+    dst = [[torch.zeros((1, w.S, h // pl.K, w.D), dtype=torch.bfloat16, device="cuda") for _ in range(w.N)]
+           for h in (w.Hq, w.Hkv, w.Hkv)]
+    basp.basp_reshard_qkv_s2h(pl, *src, *dst)
+    torch.cuda.synchronize()
+    for a, d in zip(seq, dst):
+        assert np.array_equal(np.stack([synth.bits(t.cpu()) for t in d]), oracle.s2h(a, op))
+    back = [torch.zeros_like(t) for t in src[0]]
+    basp.basp_reshard_h2s(pl, w.Hq, dst[0], back)              # the head-sharded Q stands in for O: same shape
+    torch.cuda.synchronize()
+    assert np.array_equal(np.stack([synth.bits(t.cpu()) for t in back]), seq[0])
+    assert np.array_equal(oracle.h2s(oracle.s2h(seq[0], op), op), seq[0])

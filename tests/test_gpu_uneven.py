@@ -174,3 +174,35 @@ def test_host_buffer_entry(basp):
     basp.basp_layer_fwd_host(pl, hq, hk, hv, ho, arena)
     basp.basp_get_status()
     assert_attn_close(cat(f64_list(ho)), cat(ref["o_seq"]), "host entry, uneven")
+
+
+def test_sequence_shard_right_behind_the_last_head_shard(basp):
+    """One arena with the head shards packed back to back at their exact size (whole sequences of S tokens, smaller than
+    K chunks of T tokens) and the sequence shards directly behind them: nothing overlaps, so both exchanges must accept
+    the layout, and they must be bit-exact on it."""
+    w = CASES[1]                                            # one group of 4, S = 1021: T = 256, last rank 253 tokens
+    pl = make_plan(basp, w)
+    op = oracle.plan_uneven(w.N, w.B, w.S)
+    Xq = synth.random_bits((w.B, w.S, w.Hq, w.D), seed=5)
+    seq_ref = oracle.partition_uneven(Xq, op)
+    head_ref = oracle.s2h_uneven(seq_ref, op)
+    head_elems = w.S * (w.Hq // pl.K) * w.D
+    seq_elems = [a.size for a in seq_ref]
+    arena = torch.zeros(w.N * head_elems + sum(seq_elems), dtype=torch.bfloat16, device="cuda")
+    heads = [arena[r * head_elems:(r + 1) * head_elems] for r in range(w.N)]
+    seqs, off = [], w.N * head_elems
+    for n in seq_elems:
+        seqs.append(arena[off:off + n])
+        off += n
+    assert seqs[0].data_ptr() == heads[-1].data_ptr() + head_elems * 2
+    for t, a in zip(seqs, seq_ref):
+        t.copy_(synth.from_bits(a).reshape(-1))
+    basp.basp_reshard_s2h(pl, w.Hq, seqs, heads)
+    torch.cuda.synchronize()
+    assert np.array_equal(np.stack([synth.bits(h.cpu()).reshape(head_ref[r].shape) for r, h in enumerate(heads)]), head_ref)
+    for t in seqs:
+        t.zero_()
+    basp.basp_reshard_h2s(pl, w.Hq, heads, seqs)
+    torch.cuda.synchronize()
+    for t, a in zip(seqs, seq_ref):
+        assert np.array_equal(synth.bits(t.cpu()).reshape(a.shape), a)

@@ -139,3 +139,43 @@ def test_null_and_alignment_checks_need_no_gpu(basp):
     pl3 = basp.basp_plan_create(4, 2, 1024, 8, 8, 40)    # head dim the kernels do not implement (not a multiple of 16)
     assert L.basp_attn_fwd(pl3.handle, good, good, good, good2, None, 0.0, None) == basp.BASP_ERR_UNSUPPORTED
     assert basp.lib.basp_strerror(-7).decode().startswith("a bounded wait")
+
+
+def test_scale_checks_need_no_gpu(basp):
+    """A negative, infinite or NaN softmax scale is refused by every call that takes one, before anything is launched."""
+    import ctypes
+    pl = basp.basp_plan_create(4, 2, 1024, 8, 8, 64)
+    a = (ctypes.c_void_p * 4)(*[0x10000 * (i + 1) for i in range(4)])
+    b = (ctypes.c_void_p * 4)(*[0x10000000 + 0x100000 * (i + 1) for i in range(4)])
+    ws = ctypes.c_void_p(0x40000000)
+    L = basp.lib
+    for bad in (-0.125, float("inf"), float("nan")):
+        assert L.basp_attn_fwd(pl.handle, a, a, a, b, None, bad, None) == basp.BASP_ERR_INVALID
+        assert L.basp_layer_fwd_fused(pl.handle, a, a, a, b, None, bad, None) == basp.BASP_ERR_INVALID
+        assert L.basp_layer_fwd(pl.handle, a, a, a, b, None, ws, 1 << 30, bad, None) == basp.BASP_ERR_INVALID
+        assert L.basp_attn_bwd(pl.handle, a, a, a, a, a, a, b, b, b, ws, 1 << 30, bad, None) == basp.BASP_ERR_INVALID
+        assert L.basp_layer_bwd(pl.handle, a, a, a, a, a, a, b, b, b, ws, 1 << 30, bad, None) == basp.BASP_ERR_INVALID
+
+
+def test_uneven_head_shards_may_touch_the_next_buffer(basp):
+    """Where the group size does not divide the sequence length a head-sharded shard (whole sequences of S tokens) is
+    smaller than K full chunks: a buffer that starts right behind the last head shard does not overlap it."""
+    import ctypes
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("made-up addresses: with a device present the accepted call would launch on them "
+                    "(tests/test_gpu_uneven.py covers the case on real buffers)")
+    N, S, H, D = 4, 1021, 8, 64                           # one group of 4: T = 256, last rank 253 tokens
+    pl = basp.basp_plan_create(N, 1, S, H, H, D)
+    assert (pl.K, pl.T, pl.T_last) == (4, 256, 253)
+    head_bytes = S * (H // 4) * D * 2                     # exact size of a head shard
+    seq_bytes = 256 * H * D * 2
+    heads = [0x20000000 + r * head_bytes for r in range(N)]
+    behind = heads[-1] + head_bytes                       # the first byte after the last head shard (16-byte aligned)
+    assert behind % 16 == 0
+    seqs = [behind + r * seq_bytes for r in range(N)]
+    P = lambda xs: (ctypes.c_void_p * N)(*xs)
+    rc = basp.lib.basp_reshard_h2s(pl.handle, H, P(heads), P(seqs), None)
+    assert rc in (basp.BASP_OK, basp.BASP_ERR_CUDA)       # passed the overlap check (no GPU here: the launch may fail)
+    seqs[0] -= 16                                         # one vector into the last head shard: a real overlap
+    assert basp.lib.basp_reshard_h2s(pl.handle, H, P(heads), P(seqs), None) == basp.BASP_ERR_ALIAS
