@@ -455,13 +455,14 @@ def run_gpu(args, w: synth.Workload):
         shape = Shape(basp, w, dev, seed=1000 + rank)
         t = time_steps(shape, args.steps, args.warmup, rank, local_rank)
         proj = time_projections(basp, shape, args, dev) if args.proj else None
+        ms_fused = time_fused(shape, args.steps, args.warmup) if (args.fused and not w.train) else None
         if rank == 0:
             k = rates(w, t, peaks)
             print(json.dumps({"workload": w.name, "ms_per_step": t["total_ms"] / args.steps, "ms_s2h": t["ms_s2h"],
                               "ms_attn": t["ms_attn"], "ms_h2s": t["ms_h2s"], "gpu_launches": t["launches"],
                               "attn_tflops": k["attn_fwd"]["tflops"], "clocks": t["clocks"],
                               "bwd_ms_s2h_attn_h2s": [t["ms_s2h_do"], t["ms_attn_bwd"], t["ms_h2s_grads"]] if w.train else None,
-                              "projections": proj,
+                              "projections": proj, "ms_fused": ms_fused,
                               "attn_bwd_tflops": k["attn_bwd"]["tflops"] if w.train else None}), flush=True)
         pdist.finalize()
         return
@@ -580,6 +581,7 @@ def main():
     ap.add_argument("--impl", default="basp", choices=["basp", "reference"])
     ap.add_argument("--proj", action="store_true", help="also time the QKV and output projection GEMMs (with --quick)")
     ap.add_argument("--quick", action="store_true", help="time the kernels of one shape only (for profiler runs)")
+    ap.add_argument("--fused", action="store_true", help="with --quick: also time basp_layer_fwd_fused after the three launches")
     ap.add_argument("--no-configs", action="store_true", help="the headline shape only (no `configs`, no `span`)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)

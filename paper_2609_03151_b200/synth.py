@@ -57,6 +57,7 @@ WORKLOADS = {
     "sweep_b4": Workload("sweep_b4", N=8, B=4, S=16384, Hq=32, Hkv=8, D=128),
     "sweep_b8": Workload("sweep_b8", N=8, B=8, S=8192, Hq=32, Hkv=8, D=128),
     "qwen25_7b_64k": Workload("qwen25_7b_64k", N=8, B=2, S=65536, Hq=28, Hkv=4, D=128),
+    "qwen25_7b_16k": Workload("qwen25_7b_16k", N=8, B=2, S=16384, Hq=28, Hkv=4, D=128),      # the 64K shape cut down for profiler captures
     "llama3_8b_16k_train": Workload("llama3_8b_16k_train", N=8, B=1, S=16384, Hq=32, Hkv=8, D=128, train=True),
     "llama3_8b_128k_train": Workload("llama3_8b_128k_train", N=8, B=1, S=131072, Hq=32, Hkv=8, D=128, train=True),
 }
