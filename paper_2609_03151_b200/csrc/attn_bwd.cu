@@ -162,9 +162,21 @@ __device__ __forceinline__ void bwd_report(int *status, int code, int role, int 
 #undef BWD_WAIT
 
 // Delta[bl][h][s] = sum_d O[bl][s][h][d] * dO[bl][s][h][d]; one 16-lane group per (s, h) row of D <= 128.
-__global__ void __launch_bounds__(256) bwd_delta_kernel(const __nv_bfloat16 *__restrict__ o,
-                                                        const __nv_bfloat16 *__restrict__ dout,
-                                                        float *__restrict__ delta, int Bl, int S, int H, int D) {
+template <int R>
+struct BwdHelperPtrs {
+    const __nv_bfloat16 *o[R], *dout[R];
+    float *delta[R];
+    const float *acc[R];
+    __nv_bfloat16 *dq[R];
+};
+
+// (one launch for every rank: blockIdx.y = rank)
+template <int R>
+__global__ void __launch_bounds__(256) bwd_delta_kernel(const __grid_constant__ BwdHelperPtrs<R> hp, int Bl, int S, int H,
+                                                        int D) {
+    const __nv_bfloat16 *__restrict__ o = hp.o[blockIdx.y];
+    const __nv_bfloat16 *__restrict__ dout = hp.dout[blockIdx.y];
+    float *__restrict__ delta = hp.delta[blockIdx.y];
     constexpr int lanes = 16;                           // threads per row (16 bytes each; D / 8 of them have data)
     const long long rows = (long long)Bl * S * H;
     const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -189,8 +201,10 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const __nv_bfloat16 *__r
 }
 
 // bf16(dQ accumulator), 8 elements per thread.
-__global__ void __launch_bounds__(256) bwd_dq_convert_kernel(const float *__restrict__ acc,
-                                                             __nv_bfloat16 *__restrict__ out, long long n8) {
+template <int R>
+__global__ void __launch_bounds__(256) bwd_dq_convert_kernel(const __grid_constant__ BwdHelperPtrs<R> hp, long long n8) {
+    const float *__restrict__ acc = hp.acc[blockIdx.y];
+    __nv_bfloat16 *__restrict__ out = hp.dq[blockIdx.y];
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n8) return;
     const float4 a = reinterpret_cast<const float4 *>(acc)[2 * i], b = reinterpret_cast<const float4 *>(acc)[2 * i + 1];
@@ -241,11 +255,15 @@ int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, 
 
     if (!two_pass) BASP_CUDA_TRY(cudaMemsetAsync(acc0, 0, (size_t)pl->N * acc_b, st));
     const long long row_threads = (long long)pl->Bl * pl->S * pl->Hq_l * 16;
+    BwdHelperPtrs<R> hp;
     for (int r = 0; r < pl->N; ++r) {
-        bwd_delta_kernel<<<(unsigned)((row_threads + 255) / 256), 256, 0, st>>>(
-            (const __nv_bfloat16 *)o[r], (const __nv_bfloat16 *)dout[r], const_cast<float *>(prm.delta[r]), pl->Bl,
-            pl->S, pl->Hq_l, pl->D);
+        hp.o[r] = (const __nv_bfloat16 *)o[r];
+        hp.dout[r] = (const __nv_bfloat16 *)dout[r];
+        hp.delta[r] = const_cast<float *>(prm.delta[r]);
+        hp.acc[r] = prm.dq_accp[r];
+        hp.dq[r] = (__nv_bfloat16 *)dq[r];
     }
+    bwd_delta_kernel<R><<<dim3((unsigned)((row_threads + 255) / 256), (unsigned)pl->N), 256, 0, st>>>(hp, pl->Bl, pl->S, pl->Hq_l, pl->D);
     BASP_CUDA_TRY(cudaGetLastError());
 
     int dev = 0, sms = 0;
@@ -262,7 +280,7 @@ int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, 
         const long long items_q = n_tiles * pl->N * pl->Bl * pl->Hq_l;
         attn_bwd_pass_kernel<1, R><<<(int)(items_q < sms ? items_q : sms), kBwdThreads, smem, st>>>(prm);
         BASP_CUDA_TRY(cudaGetLastError());
-        basp_count_launch(2 + pl->N);
+        basp_count_launch(3);
         return BASP_OK;
     }
     if (pl->D > 64) {        // 80 .. 128: the pipelined 128-wide kernel (attn_bwd_d128.cuh)
@@ -300,11 +318,9 @@ int bwd_launch(const basp_plan *pl, const void *const *q, const void *const *k, 
     BASP_CUDA_TRY(cudaGetLastError());
 
     const long long n8 = (long long)(acc_b / sizeof(float) / 8);
-    for (int r = 0; r < pl->N; ++r)
-        bwd_dq_convert_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>(
-            reinterpret_cast<const float *>(reinterpret_cast<const char *>(acc0) + (size_t)r * acc_b), (__nv_bfloat16 *)dq[r], n8);
+    bwd_dq_convert_kernel<R><<<dim3((unsigned)((n8 + 255) / 256), (unsigned)pl->N), 256, 0, st>>>(hp, n8);
     BASP_CUDA_TRY(cudaGetLastError());
-    basp_count_launch(1 + 2 * pl->N);
+    basp_count_launch(3);
     return BASP_OK;
 }
 
