@@ -219,6 +219,16 @@ class Shape:
             self.lse = [torch.empty((Bl, plan.Hq_l, w.S), dtype=torch.float32, device=dev) for _ in range(N)]
             self.bwd_ws = torch.empty(basp.basp_attn_bwd_workspace_bytes(plan), dtype=torch.uint8, device=dev)
         self.n_events = 7 if w.train else 4
+        self.seed = seed
+
+    def checksum(self) -> dict:
+        """Sum of the bf16 bit patterns of every input shard (what identifies the drawn inputs of a run)."""
+        tot = lambda ts: int(sum(int(t.view(torch.int16).to(torch.int64).sum().item()) for t in ts))
+        out = {"generator": f"torch device generator, seed {self.seed}, N(0,1) in fp32 rounded to bf16, per shard in the order Q, K, V",
+               "q": tot(self.q_seq), "k": tot(self.k_seq), "v": tot(self.v_seq)}
+        if self.w.train:
+            out["do"] = tot(self.do_seq)
+        return out
 
     def step(self, events=None):
         """a2 -> a3 -> a4 (what basp_layer_fwd launches) and, for a training workload, a7 -> a6 -> a7 (what
@@ -469,6 +479,7 @@ def run_gpu(args, w: synth.Workload):
 
     # ---- the headline shape: exactly args.steps timed steps after args.warmup untimed ones
     shape = Shape(basp, w, dev, seed=1000 + rank)
+    inputs = shape.checksum()
     t = time_steps(shape, args.steps, args.warmup, rank, local_rank)
     ms_per_step = pdist.max_over_ranks(t["total_ms"] / args.steps)
     k = rates(w, t, peaks)
@@ -518,7 +529,7 @@ def run_gpu(args, w: synth.Workload):
             "metric": METRIC, "value": tokens_all / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": config_dict(w), "clocks": t["clocks"], "e2e": e2e, "gpu_launches": t["launches"],
+            "config": config_dict(w), "inputs": inputs, "clocks": t["clocks"], "e2e": e2e, "gpu_launches": t["launches"],
             "ms_per_step_median": statistics.median(t["per_step"]), "ms_per_step_best": min(t["per_step"]),
             "roofline": {"kernel": top_name, "bound": "tensor", "achieved": top["tflops"], "peak": peaks["bf16_sustained"],
                          "unit": "TFLOP/s", "frac": top["frac_of_sustained"], "traffic": ncu_traffic(w.name, top_name),

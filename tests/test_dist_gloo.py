@@ -220,3 +220,37 @@ def test_two_process_multi_gpu_layer_ordering(tmp_path):
     port = _free_port()
     mp.spawn(_worker_multi_gpu_order, args=(2, port, str(tmp_path)), nprocs=2, join=True)
     assert all((tmp_path / f"order{r}").exists() for r in range(2))
+
+
+def test_three_step_multi_gpu_host_ordering():
+    """The three-step group-spanning layer on one process with stand-ins: every step is launched on the given stream and
+    followed by a synchronisation of that stream and a barrier (a step reads what other GPUs wrote in the step before),
+    with this GPU's rank range and the eight shard tables."""
+    n_ranks, world, gpu = 8, 4, 1
+    sizes = {n: 4096 for n in ("q", "k", "v", "o", "qh", "kh", "vh", "oh")}
+    sh = pdist.SymmetricShards(n_ranks, sizes, allocator=_cpu_allocator(world, gpu), world=world, gpu=gpu)
+    log = []
+
+    class Plan:
+        Hq = 32
+
+    class StubBinding:
+        @staticmethod
+        def basp_reshard_qkv_s2h_ranks(plan, q, k, v, qh, kh, vh, r0, cnt, stream=None):
+            assert (q, qh, vh) == (sh.addresses("q"), sh.addresses("qh"), sh.addresses("vh"))
+            log.append(("s2h", stream.name, r0, cnt))
+
+        @staticmethod
+        def basp_attn_fwd_ranks(plan, qh, kh, vh, oh, r0, cnt, lse_shards=None, softmax_scale=0.0, stream=None):
+            assert (kh, oh) == (sh.addresses("kh"), sh.addresses("oh"))
+            log.append(("attn", stream.name, r0, cnt))
+
+        @staticmethod
+        def basp_reshard_h2s_ranks(plan, n_heads, oh, o, r0, cnt, stream=None):
+            assert n_heads == 32 and (oh, o) == (sh.addresses("oh"), sh.addresses("o"))
+            log.append(("h2s", stream.name, r0, cnt))
+
+    s = _RecordingStream(log, "s")
+    pdist.layer_fwd_three_step_multi_gpu(Plan, sh, stream=s, binding=StubBinding, barrier=lambda: log.append(("barrier",)))
+    sync_bar = [("sync", "s"), ("barrier",)]
+    assert log == sync_bar + [("s2h", "s", 2, 2)] + sync_bar + [("attn", "s", 2, 2)] + sync_bar + [("h2s", "s", 2, 2)] + sync_bar
