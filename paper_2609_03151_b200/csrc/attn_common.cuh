@@ -31,6 +31,7 @@ struct AttnParams {
     // divisors of the item decoding, prepared on the host (a division by a runtime value is some 25 instructions, and
     // the decoding is inlined into every role: instruction fetch matters in this kernel)
     FastDiv div_per_band, div_per_stream, div_q_per_kv, div_hkv_l, div_bl;
+    FastDiv div_T, div_K;   // of the fused tile addressing (owner rank of a sequence position, group of a rank)
 };
 
 struct TileCoord {
@@ -44,8 +45,8 @@ __device__ __forceinline__ TileCoord locate(const AttnParams<R> &p, int r, int b
                                             int rep = 1) {
     TileCoord c;
     if (p.fused) {
-        const int g = r / p.K, l = r - g * p.K;
-        const int owner = s0 / p.T;
+        const int g = (int)fdiv((uint32_t)r, p.div_K), l = r - g * p.K;
+        const int owner = (int)fdiv((uint32_t)s0, p.div_T);
         c.rank = g * p.K + owner;
         c.row = bl * p.T + (s0 - owner * p.T);
         c.head = rep > 1 ? l / rep : l * heads_l + h;

@@ -58,6 +58,8 @@ int fill_and_launch(const basp_plan *pl, const void *const *q, const void *const
         prm.div_q_per_kv = make_fastdiv((uint32_t)q_per_kv);
         prm.div_hkv_l = make_fastdiv((uint32_t)pl->Hkv_l);
         prm.div_bl = make_fastdiv((uint32_t)pl->Bl);
+        prm.div_T = make_fastdiv((uint32_t)pl->T);
+        prm.div_K = make_fastdiv((uint32_t)pl->K);
     }
     prm.fused = fused; prm.causal = pl->causal; prm.has_lse = lse != nullptr;
     prm.scale_log2 = (scale == 0.f ? 1.f / sqrtf((float)pl->D) : scale) * 1.4426950408889634f;
