@@ -516,7 +516,12 @@ def run_gpu(args, w: synth.Workload):
             ww = synth.WORKLOADS[name]
             configs[name] = measure_shape(basp, ww, dev, rank, local_rank, 3 if ww.train else min(args.steps, 10),
                                           max(3, min(args.warmup, 5)), peaks)
-    span = measure_span(basp, dev, rank, world, max(2, min(args.steps, 10)), args.warmup) if not args.no_configs else None
+    span = None
+    if not args.no_configs:
+        try:
+            span = measure_span(basp, dev, rank, world, max(2, min(args.steps, 10)), args.warmup)
+        except Exception as e:      # the group-spanning leg must not take the headline number down with it (it needs
+            span = {"error": f"{type(e).__name__}: {e}"[:300]}       # symmetric memory across the run's GPUs)
 
     if rank == 0:
         cpu = None
